@@ -1,0 +1,189 @@
+/*
+ * gnnpre — multi-hop feature aggregation  X_k = A^ X_{k-1}, k = 1..K, on one Blackwell GPU.
+ *
+ * C ABI of libgnnpre.so.  The library implements the block-wise precomputation of
+ * arXiv 2207.12000, Section 3.2 ("Efficient Precomputation"):
+ *   - the edge list E of the operator's support is cut into b disjoint, balanced sets
+ *     ("Precomputation on GPU", Eq. 10; Algorithm 1, the split of S),
+ *   - the feature matrix is cut into c column slabs (Algorithm 1, the split of X_prev),
+ *   - (b, c) minimise b*c under a device-memory budget (Eq. 12),
+ *   - every hop multiplies the previous hop (Algorithm 1's outer loop); all K hops are kept.
+ * A^ is a constant linear filter fixed before precomputation (Section 3.1, "Limitation"):
+ *   GCN_SYM    S = D~^{-1/2} (A + I) D~^{-1/2}           (Eq. 1)
+ *   SAGE_MEAN  D^{-1} A, zero rows where D_i = 0
+ *   GIN_SUM    A + (1 + eps) I, eps fixed by the caller
+ *
+ * Conventions
+ *   - Every function returns a gnnpre_status_t (0 = success, negative = error); nothing
+ *     throws or aborts across this boundary.  On error no output argument is valid unless
+ *     stated otherwise.
+ *   - "device" pointers are CUDA device addresses on the current device; "host" pointers are
+ *     ordinary process addresses.  The library never takes ownership of a caller's buffer.
+ *   - There is no CPU fallback: host-resident operands are streamed through the GPU.
+ *   - Only sm_100 devices are accepted (GNNPRE_ERR_UNSUPPORTED_ARCH otherwise).
+ */
+#ifndef GNNPRE_H
+#define GNNPRE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GNNPRE_OK = 0,
+    GNNPRE_ERR_INVALID_ARG = -1,      /* NULL pointer, bad enum, bad size, b > |E| ... */
+    GNNPRE_ERR_INVALID_CSR = -2,      /* see gnnpre_csr_t */
+    GNNPRE_ERR_ALIGN = -3,            /* pointer not 16-byte aligned, or a leading dimension / F not a multiple of 4 */
+    GNNPRE_ERR_OOM_DEVICE = -4,
+    GNNPRE_ERR_OOM_HOST = -5,
+    GNNPRE_ERR_BUDGET_TOO_SMALL = -6, /* Eq. 12 has no feasible (b, c) */
+    GNNPRE_ERR_CUDA = -7,             /* a CUDA call failed; gnnpre_last_cuda_error() names it */
+    GNNPRE_ERR_TIMEOUT = -8,
+    GNNPRE_ERR_BUSY = -9,             /* the plan is already inside a propagate call */
+    GNNPRE_ERR_UNSUPPORTED_ARCH = -10
+} gnnpre_status_t;
+
+typedef enum { GNNPRE_OP_GCN_SYM = 0, GNNPRE_OP_SAGE_MEAN = 1, GNNPRE_OP_GIN_SUM = 2 } gnnpre_op_t;
+typedef enum { GNNPRE_MEM_DEVICE = 0, GNNPRE_MEM_HOST = 1 } gnnpre_mem_t;
+
+/*
+ * The adjacency matrix A in {0,1}^{n x n} (Section 2) in CSR form, WITHOUT diagonal entries.
+ *   rowptr[n+1] int64, rowptr[0] = 0, non-decreasing, rowptr[n] = nnz
+ *   colidx[nnz] int32, 0 <= col < n < 2^31, strictly ascending inside a row, col != row
+ * Both arrays live where `mem` says (both on the device, or both on the host; host arrays are
+ * read fastest when page-locked).  Symmetry is the caller's business: degrees are row counts.
+ * The arrays are only read during gnnpre_build_plan and may be released afterwards.
+ */
+typedef struct {
+    int64_t n;
+    int64_t nnz;
+    const int64_t* rowptr;
+    const int32_t* colidx;
+    int32_t mem; /* gnnpre_mem_t */
+} gnnpre_csr_t;
+
+/* gnnpre_plan_opts_t.flags */
+#define GNNPRE_FLAG_LAUNCH_PER_BLOCK 1u /* device-resident runs: one kernel launch per edge block instead of one per hop */
+#define GNNPRE_FLAG_SKIP_VALIDATION 2u  /* trust the CSR contract (saves one pass over the graph) */
+
+typedef struct {
+    int32_t op;              /* gnnpre_op_t */
+    float gin_eps;           /* GIN_SUM only */
+    int64_t feat_dim;        /* F: columns of X; must be a multiple of 4 */
+    int64_t budget_bytes;    /* B_GPU of Eq. 12; 0 = the device's free memory at plan time */
+    int32_t force_blocks;    /* b; 0 = solve Eq. 12 */
+    int32_t force_col_slabs; /* c; 0 = solve Eq. 12 */
+    int32_t segment_edges;   /* edges per warp-level segment; 0 = chosen from F */
+    int32_t operands_mem;    /* gnnpre_mem_t: where X and out[] will live at propagate time; HOST makes
+                                Eq. 12 count the library's four slab buffers (beta_X = 4) instead of two */
+    uint32_t flags;
+} gnnpre_plan_opts_t;
+
+typedef struct gnnpre_plan gnnpre_plan_t; /* opaque; owns device (and pinned host) memory */
+
+typedef struct {
+    int64_t n, nnz, nnz_tilde; /* nnz_tilde = |E|: nnz + n for GCN/GIN (self-loops are edges of E), nnz for SAGE */
+    int64_t feat_dim;
+    int32_t op;
+    int32_t b, c;              /* Eq. 12's block counts in use */
+    int64_t slab_width;        /* columns per slab: 4 * ceil(F / (4c)) */
+    int64_t B_S, B_X, B_fixed; /* Eq. 12's volumes in bytes: 4*nnz_tilde + 8*(n+1); 4*n*F; 16*n (per-node arrays) */
+    int64_t beta_S, beta_X;    /* Eq. 12's coefficients as this library sets them */
+    int64_t budget_bytes;
+    int64_t device_bytes;      /* device memory the plan holds */
+    int64_t host_bytes;        /* pinned host memory the plan holds */
+    int64_t num_segments;      /* warp-level edge segments over all blocks */
+    int64_t num_row_fixups;    /* rows whose edges span more than one segment */
+    int64_t num_scratch_rows;  /* partial-sum rows of scratch memory (slab_width floats each) */
+    int32_t segment_edges;
+    int32_t structure_mem;     /* gnnpre_mem_t: where the plan's copy of E lives */
+} gnnpre_plan_info_t;
+
+/* One edge block E^(l): edges [e_lo, e_hi) of the CSR-ordered edge list of the support. */
+typedef struct {
+    int64_t e_lo, e_hi;
+    int32_t row_lo, row_hi;      /* rows holding edge e_lo and edge e_hi - 1 */
+    int32_t first_row_partial;   /* row_lo also has edges in block l-1 */
+    int32_t last_row_partial;    /* row_hi also has edges in block l+1 */
+} gnnpre_block_info_t;
+
+#define GNNPRE_MAX_HOPS 64
+
+typedef struct {
+    float hop_ms[GNNPRE_MAX_HOPS]; /* device time per hop (CUDA events); device-resident runs with stats only */
+    float total_ms;
+    int64_t h2d_bytes, d2h_bytes;  /* streamed runs */
+    int64_t kernel_launches;
+} gnnpre_stats_t;
+
+/*
+ * Degrees D_i = number of nonzeros of row i (Section 2).  `deg_out` (int32[n]) lives in the same
+ * memory space as the CSR.  Device data: asynchronous on `stream`.  Host data: the row pointers
+ * travel through the GPU and the call returns when deg_out is complete.  Integer, exact.
+ */
+int gnnpre_degrees(const gnnpre_csr_t* csr, int32_t* deg_out, void* stream);
+
+/*
+ * Builds the decomposition plan (Section 3.2): validates the CSR, computes degrees (or takes the
+ * caller's `degrees`, int32[n] in the CSR's memory space; NULL = compute), the per-node scale
+ * factors of the operator (fp64 arithmetic rounded once to fp32), the edge list E of the support
+ * with self-loops inserted at their sorted position, (b, c) from Eq. 12 unless forced, the b
+ * balanced contiguous edge blocks  [floor(l|E|/b), floor((l+1)|E|/b))  and the warp-level segment
+ * tables.  Synchronous.  The plan is immutable afterwards; free it with gnnpre_plan_destroy.
+ * Errors: INVALID_ARG (NULLs, bad op, F < 4, b > |E|, c > ceil(F/4)), ALIGN (F % 4 != 0),
+ * INVALID_CSR, BUDGET_TOO_SMALL, OOM_*, CUDA, UNSUPPORTED_ARCH.
+ */
+int gnnpre_build_plan(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpre_plan_opts_t* opts,
+                      gnnpre_plan_t** plan_out);
+
+int gnnpre_plan_info(const gnnpre_plan_t* plan, gnnpre_plan_info_t* info_out);
+
+/* Block l in [0, b).  INVALID_ARG outside that range. */
+int gnnpre_plan_block(const gnnpre_plan_t* plan, int32_t l, gnnpre_block_info_t* block_out);
+
+/* Host copies for parity checks: degrees int32[n], scales fp32[n] each (A^_ij = rscale_i * cscale_j,
+ * times 1 + eps on the GIN diagonal).  Any pointer may be NULL. */
+int gnnpre_plan_scales(const gnnpre_plan_t* plan, int32_t* deg_out, float* rscale_out, float* cscale_out);
+
+/* Host copy of the support's CSR: rowptr_out int64[n+1], colidx_out int32[nnz_tilde].  Either may be NULL. */
+int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t* colidx_out);
+
+/*
+ * Algorithm 1: out[k-1] <- A^ applied k times to X, for k = 1..K (X itself is not repeated).
+ *   X      fp32 row-major [n, F] with leading dimension ldx (floats), in x_mem
+ *   out    host array of K pointers, each fp32 row-major [n, F] with leading dimension ldo, in out_mem
+ *   ldx, ldo >= F and multiples of 4; all base pointers 16-byte aligned (else GNNPRE_ERR_ALIGN)
+ *   out[k] must not overlap X or another out[]; 1 <= K <= GNNPRE_MAX_HOPS
+ * Device X and device out: the work is enqueued on `stream` and the call returns at once; the
+ * plan's scratch memory is in use until that work completes, so calls on one plan must not
+ * overlap on the GPU (use one stream per plan).
+ * Any host operand: column slabs of X travel host->device, finished output rows travel
+ * device->host on side streams while later blocks compute, and the call returns when out[] is
+ * complete in host memory (GNNPRE_ERR_BUSY if another streamed call holds the plan).  Host buffers
+ * should be page-locked for full link speed.
+ * Accumulation is fp32 in a fixed order: results are bitwise reproducible from run to run for a
+ * given plan, and agree across different (b, c) or segment sizes only to rounding.
+ * `stats` may be NULL; when given, device-resident calls synchronise `stream` to read the timers.
+ */
+int gnnpre_propagate(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t x_mem, int32_t K, float* const* out,
+                     int64_t ldo, int32_t out_mem, void* stream, gnnpre_stats_t* stats);
+
+void gnnpre_plan_destroy(gnnpre_plan_t* plan);
+
+/* Eq. 12 on its own (exposed for parity with the exhaustive search):
+ * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;
+ * ties towards smaller c, then smaller b.  BUDGET_TOO_SMALL if infeasible.  Host only. */
+int gnnpre_solve_budget(int64_t B_S, int64_t B_X, int64_t B_fixed, int64_t beta_S, int64_t beta_X, int64_t B_GPU,
+                        int64_t max_b, int64_t max_c, int64_t* b_out, int64_t* c_out);
+
+const char* gnnpre_status_string(int status);
+
+/* Text of the last CUDA error this thread saw inside the library ("" if none). */
+const char* gnnpre_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GNNPRE_H */

@@ -1,0 +1,236 @@
+"""ctypes binding of libgnnpre.so: one Python function per C entry point, same names.
+
+Only argument marshalling happens here.  Tensors are torch tensors used as plain device (or
+host) memory; every step of the computation runs inside the library's CUDA kernels.  If the
+library has not been built, importing this module raises: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Sequence
+
+import torch
+
+from . import build as _build
+
+GNNPRE_OP_GCN_SYM, GNNPRE_OP_SAGE_MEAN, GNNPRE_OP_GIN_SUM = 0, 1, 2
+GNNPRE_MEM_DEVICE, GNNPRE_MEM_HOST = 0, 1
+GNNPRE_FLAG_LAUNCH_PER_BLOCK, GNNPRE_FLAG_SKIP_VALIDATION = 1, 2
+GNNPRE_MAX_HOPS = 64
+
+
+class gnnpre_csr_t(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int64), ("nnz", ctypes.c_int64), ("rowptr", ctypes.c_void_p),
+                ("colidx", ctypes.c_void_p), ("mem", ctypes.c_int32)]
+
+
+class gnnpre_plan_opts_t(ctypes.Structure):
+    _fields_ = [("op", ctypes.c_int32), ("gin_eps", ctypes.c_float), ("feat_dim", ctypes.c_int64),
+                ("budget_bytes", ctypes.c_int64), ("force_blocks", ctypes.c_int32),
+                ("force_col_slabs", ctypes.c_int32), ("segment_edges", ctypes.c_int32),
+                ("operands_mem", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class gnnpre_plan_info_t(ctypes.Structure):
+    _fields_ = [("n", ctypes.c_int64), ("nnz", ctypes.c_int64), ("nnz_tilde", ctypes.c_int64),
+                ("feat_dim", ctypes.c_int64), ("op", ctypes.c_int32), ("b", ctypes.c_int32), ("c", ctypes.c_int32),
+                ("slab_width", ctypes.c_int64), ("B_S", ctypes.c_int64), ("B_X", ctypes.c_int64),
+                ("B_fixed", ctypes.c_int64), ("beta_S", ctypes.c_int64), ("beta_X", ctypes.c_int64),
+                ("budget_bytes", ctypes.c_int64), ("device_bytes", ctypes.c_int64), ("host_bytes", ctypes.c_int64),
+                ("num_segments", ctypes.c_int64), ("num_row_fixups", ctypes.c_int64),
+                ("num_scratch_rows", ctypes.c_int64), ("segment_edges", ctypes.c_int32),
+                ("structure_mem", ctypes.c_int32)]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class gnnpre_block_info_t(ctypes.Structure):
+    _fields_ = [("e_lo", ctypes.c_int64), ("e_hi", ctypes.c_int64), ("row_lo", ctypes.c_int32),
+                ("row_hi", ctypes.c_int32), ("first_row_partial", ctypes.c_int32),
+                ("last_row_partial", ctypes.c_int32)]
+
+
+class gnnpre_stats_t(ctypes.Structure):
+    _fields_ = [("hop_ms", ctypes.c_float * GNNPRE_MAX_HOPS), ("total_ms", ctypes.c_float),
+                ("h2d_bytes", ctypes.c_int64), ("d2h_bytes", ctypes.c_int64), ("kernel_launches", ctypes.c_int64)]
+
+
+class GnnpreError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        text = _lib.gnnpre_status_string(status).decode()
+        detail = _lib.gnnpre_last_cuda_error().decode()
+        super().__init__(f"{where}: {text} ({status})" + (f" [{detail}]" if detail and status == -7 else ""))
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: run paper_2207_12000_b200.build.build() (needs nvcc); "
+                          "there is no fallback implementation")
+    lib = ctypes.CDLL(path)
+    p, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    lib.gnnpre_degrees.argtypes = [ctypes.POINTER(gnnpre_csr_t), p, p]
+    lib.gnnpre_build_plan.argtypes = [ctypes.POINTER(gnnpre_csr_t), p, ctypes.POINTER(gnnpre_plan_opts_t),
+                                      ctypes.POINTER(p)]
+    lib.gnnpre_plan_info.argtypes = [p, ctypes.POINTER(gnnpre_plan_info_t)]
+    lib.gnnpre_plan_block.argtypes = [p, i32, ctypes.POINTER(gnnpre_block_info_t)]
+    lib.gnnpre_plan_scales.argtypes = [p, p, p, p]
+    lib.gnnpre_plan_support.argtypes = [p, p, p]
+    lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
+                                     ctypes.POINTER(gnnpre_stats_t)]
+    lib.gnnpre_plan_destroy.argtypes = [p]
+    lib.gnnpre_plan_destroy.restype = None
+    lib.gnnpre_solve_budget.argtypes = [i64] * 8 + [ctypes.POINTER(i64), ctypes.POINTER(i64)]
+    lib.gnnpre_status_string.argtypes = [ctypes.c_int]
+    lib.gnnpre_status_string.restype = ctypes.c_char_p
+    lib.gnnpre_last_cuda_error.restype = ctypes.c_char_p
+    return lib
+
+
+_lib = _load()
+
+
+def _check(status: int, where: str) -> None:
+    if status != 0:
+        raise GnnpreError(status, where)
+
+
+def _mem_of(t: torch.Tensor) -> int:
+    return GNNPRE_MEM_DEVICE if t.is_cuda else GNNPRE_MEM_HOST
+
+
+def _csr(rowptr: torch.Tensor, colidx: torch.Tensor) -> gnnpre_csr_t:
+    assert rowptr.dtype == torch.int64 and colidx.dtype == torch.int32
+    assert rowptr.is_contiguous() and colidx.is_contiguous() and rowptr.device == colidx.device
+    return gnnpre_csr_t(rowptr.numel() - 1, colidx.numel(), rowptr.data_ptr(), colidx.data_ptr(), _mem_of(rowptr))
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def gnnpre_degrees(rowptr: torch.Tensor, colidx: torch.Tensor, stream=None) -> torch.Tensor:
+    csr = _csr(rowptr, colidx)
+    deg = torch.empty(csr.n, dtype=torch.int32, device=rowptr.device)
+    _check(_lib.gnnpre_degrees(ctypes.byref(csr), deg.data_ptr(), _stream_ptr(stream)), "gnnpre_degrees")
+    return deg
+
+
+class Plan:
+    """Owns a gnnpre_plan_t*; destroyed with the object."""
+
+    def __init__(self, handle: int, keepalive):
+        self._h = ctypes.c_void_p(handle)
+        self._keepalive = keepalive
+
+    @property
+    def handle(self):
+        return self._h
+
+    def info(self) -> dict:
+        return gnnpre_plan_info(self)
+
+    def close(self):
+        if self._h:
+            _lib.gnnpre_plan_destroy(self._h)
+            self._h = ctypes.c_void_p(None)
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def gnnpre_build_plan(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, feat_dim: int, *, degrees=None,
+                      gin_eps: float = 0.0, budget_bytes: int = 0, force_blocks: int = 0, force_col_slabs: int = 0,
+                      segment_edges: int = 0, operands_mem: int = GNNPRE_MEM_DEVICE, flags: int = 0) -> Plan:
+    csr = _csr(rowptr, colidx)
+    opts = gnnpre_plan_opts_t(op, gin_eps, feat_dim, budget_bytes, force_blocks, force_col_slabs, segment_edges,
+                              operands_mem, flags)
+    if degrees is not None:
+        assert degrees.dtype == torch.int32 and degrees.device == rowptr.device and degrees.is_contiguous()
+    out = ctypes.c_void_p()
+    _check(_lib.gnnpre_build_plan(ctypes.byref(csr), degrees.data_ptr() if degrees is not None else None,
+                                  ctypes.byref(opts), ctypes.byref(out)), "gnnpre_build_plan")
+    return Plan(out.value, None)
+
+
+def gnnpre_plan_info(plan: Plan) -> dict:
+    info = gnnpre_plan_info_t()
+    _check(_lib.gnnpre_plan_info(plan.handle, ctypes.byref(info)), "gnnpre_plan_info")
+    return info.as_dict()
+
+
+def gnnpre_plan_block(plan: Plan, l: int) -> dict:
+    blk = gnnpre_block_info_t()
+    _check(_lib.gnnpre_plan_block(plan.handle, l, ctypes.byref(blk)), "gnnpre_plan_block")
+    return {k: getattr(blk, k) for k, _ in blk._fields_}
+
+
+def gnnpre_plan_scales(plan: Plan):
+    """(degrees int32, rscale fp32, cscale fp32) as host tensors."""
+    n = gnnpre_plan_info(plan)["n"]
+    deg = torch.empty(n, dtype=torch.int32)
+    r = torch.empty(n, dtype=torch.float32)
+    c = torch.empty(n, dtype=torch.float32)
+    _check(_lib.gnnpre_plan_scales(plan.handle, deg.data_ptr(), r.data_ptr(), c.data_ptr()), "gnnpre_plan_scales")
+    return deg, r, c
+
+
+def gnnpre_plan_support(plan: Plan):
+    """(rowptr int64 [n+1], colidx int32 [nnz_tilde]) of the operator's support, as host tensors."""
+    info = gnnpre_plan_info(plan)
+    rp = torch.empty(info["n"] + 1, dtype=torch.int64)
+    ci = torch.empty(info["nnz_tilde"], dtype=torch.int32)
+    _check(_lib.gnnpre_plan_support(plan.handle, rp.data_ptr(), ci.data_ptr()), "gnnpre_plan_support")
+    return rp, ci
+
+
+def gnnpre_propagate(plan: Plan, X: torch.Tensor, K: int, out: Sequence[torch.Tensor] | None = None, *,
+                     stream=None, want_stats: bool = False):
+    """out[k-1] = A^ applied k times to X.  X and out are fp32 row-major views (stride(1) == 1) on the
+    device, or host tensors (preferably pinned) for the streamed path.  Returns (out, stats-or-None)."""
+    assert X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    n, F = X.shape
+    if out is None:
+        if X.is_cuda:
+            out = [torch.empty((n, F), dtype=torch.float32, device=X.device) for _ in range(K)]
+        else:
+            out = [torch.empty((n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
+    assert len(out) == K
+    ldo = out[0].stride(0)
+    for o in out:
+        assert o.dtype == torch.float32 and o.shape == (n, F) and o.stride(1) == 1 and o.stride(0) == ldo
+        assert o.is_cuda == out[0].is_cuda
+    ptrs = (ctypes.c_void_p * K)(*[o.data_ptr() for o in out])
+    stats = gnnpre_stats_t() if want_stats else None
+    _check(_lib.gnnpre_propagate(plan.handle, X.data_ptr(), X.stride(0), _mem_of(X), K, ptrs, ldo, _mem_of(out[0]),
+                                 _stream_ptr(stream), ctypes.byref(stats) if want_stats else None),
+           "gnnpre_propagate")
+    return list(out), stats
+
+
+def gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
+    b, c = ctypes.c_int64(), ctypes.c_int64()
+    rc = _lib.gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c, ctypes.byref(b),
+                                  ctypes.byref(c))
+    if rc == -6:
+        return None
+    _check(rc, "gnnpre_solve_budget")
+    return b.value, c.value
+
+
+def gnnpre_status_string(status: int) -> str:
+    return _lib.gnnpre_status_string(status).decode()
+
+
+def exported_symbols():
+    return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_status_string", "gnnpre_last_cuda_error"]

@@ -1,0 +1,65 @@
+// C-ABI glue: argument checks, status text, and the dispatch of gnnpre_propagate.
+#include <cstdio>
+#include <cstring>
+
+#include "gnnpre_internal.cuh"
+
+namespace gnnpre {
+
+namespace {
+thread_local char g_last_error[512] = "";
+}
+
+void set_last_cuda_error(cudaError_t e, const char* what, const char* file, int line) {
+    const char* base = std::strrchr(file, '/');
+    std::snprintf(g_last_error, sizeof(g_last_error), "%s: %s (%s:%d)", cudaGetErrorName(e), what,
+                  base ? base + 1 : file, line);
+}
+
+}  // namespace gnnpre
+
+using namespace gnnpre;
+
+extern "C" const char* gnnpre_last_cuda_error(void) { return g_last_error; }
+
+extern "C" const char* gnnpre_status_string(int status) {
+    switch (status) {
+    case GNNPRE_OK: return "ok";
+    case GNNPRE_ERR_INVALID_ARG: return "invalid argument";
+    case GNNPRE_ERR_INVALID_CSR: return "CSR violates the input contract";
+    case GNNPRE_ERR_ALIGN: return "misaligned pointer, leading dimension or feature width";
+    case GNNPRE_ERR_OOM_DEVICE: return "out of device memory";
+    case GNNPRE_ERR_OOM_HOST: return "out of host memory";
+    case GNNPRE_ERR_BUDGET_TOO_SMALL: return "memory budget admits no (b, c)";
+    case GNNPRE_ERR_CUDA: return "CUDA error";
+    case GNNPRE_ERR_TIMEOUT: return "timed out";
+    case GNNPRE_ERR_BUSY: return "plan is busy";
+    case GNNPRE_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    default: return "unknown status";
+    }
+}
+
+extern "C" int gnnpre_propagate(gnnpre_plan_t* P, const float* X, int64_t ldx, int32_t x_mem, int32_t K,
+                                float* const* out, int64_t ldo, int32_t out_mem, void* stream, gnnpre_stats_t* stats) {
+    if (!P || !X || !out || K < 1 || K > GNNPRE_MAX_HOPS) return GNNPRE_ERR_INVALID_ARG;
+    if ((x_mem != GNNPRE_MEM_DEVICE && x_mem != GNNPRE_MEM_HOST) ||
+        (out_mem != GNNPRE_MEM_DEVICE && out_mem != GNNPRE_MEM_HOST))
+        return GNNPRE_ERR_INVALID_ARG;
+    if (ldx < P->feat_dim || ldo < P->feat_dim) return GNNPRE_ERR_INVALID_ARG;
+    if (ldx % 4 != 0 || ldo % 4 != 0 || (reinterpret_cast<uintptr_t>(X) & 15u)) return GNNPRE_ERR_ALIGN;
+    for (int32_t k = 0; k < K; ++k) {
+        if (!out[k]) return GNNPRE_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(out[k]) & 15u) return GNNPRE_ERR_ALIGN;
+        if (out[k] == X) return GNNPRE_ERR_INVALID_ARG;
+        for (int32_t j = 0; j < k; ++j)
+            if (out[j] == out[k]) return GNNPRE_ERR_INVALID_ARG;
+    }
+    if (stats) std::memset(stats, 0, sizeof(*stats));
+    int dev = -1;
+    GNNPRE_CUDA(cudaGetDevice(&dev));
+    if (dev != P->device) return GNNPRE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (x_mem == GNNPRE_MEM_DEVICE && out_mem == GNNPRE_MEM_DEVICE && P->structure_mem == GNNPRE_MEM_DEVICE)
+        return propagate_resident(P, X, ldx, K, out, ldo, st, stats);
+    return propagate_streamed(P, X, ldx, x_mem, K, out, ldo, out_mem, st, stats);
+}

@@ -1,0 +1,408 @@
+// Propagation kernels: one hop  X_out = A^ X_prev  over a range of warp-level edge segments
+// (Algorithm 1's block product Z = S^(j) X^(i) and its accumulation X_tmp += Z, fused; the
+// operator's normalisation of Eq. 1 / Eq. 10 is applied on the fly from per-node scales, so S is
+// never materialised).
+//
+// Work decomposition.  The edge list E of the support is cut, inside every edge block, into short
+// contiguous segments.  A group of G lanes (G = 4..32, so that one lane holds one or more float4 of
+// a feature row) walks one segment edge by edge: the group reads up to G column indices with one
+// coalesced load, then gathers the neighbours' feature rows with 128-bit loads, several rows in
+// flight per lane, and accumulates in fp32 registers.  Bit 31 of a column entry marks the last edge
+// of a row: there the group scales the sum by r_i and stores the output row.  Rows cut by a segment
+// boundary leave their partial sums in scratch rows, which k_row_fixups adds up in a fixed order.
+#include <algorithm>
+
+#include "gnnpre_internal.cuh"
+
+namespace gnnpre {
+
+namespace {
+
+struct SegArgs {
+    const Segment* segs;
+    int64_t seg_lo, seg_hi;
+    const uint32_t* colx;
+    int64_t colx_base;
+    const float* x;
+    int64_t ldx;
+    float* out;
+    int64_t ldo;
+    float* scratch;
+    int64_t scratch_ld;
+    const float* rscale;
+    const float* cscale;
+    const int32_t* nzrows;
+    int32_t f4;  // float4 per row of this column tile
+    float diag_weight;  // GIN: 1 + eps
+};
+
+__device__ __forceinline__ float4 ld_row(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
+
+__device__ __forceinline__ void fma4(float4& a, float w, const float4& x) {
+    a.x = fmaf(w, x.x, a.x);
+    a.y = fmaf(w, x.y, a.y);
+    a.z = fmaf(w, x.z, a.z);
+    a.w = fmaf(w, x.w, a.w);
+}
+
+constexpr int kThreads = 256;
+
+// G lanes per segment, V float4 per lane (row width <= 4*G*V floats), U rows in flight per lane.
+template <int G, int V, int U, int OP, bool HAS_EMPTY>
+__global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
+    constexpr unsigned kFull = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (G - 1);
+    const int gshift = lane & ~(G - 1);
+    const unsigned glow = G == 32 ? kFull : ((1u << G) - 1u);
+    const unsigned gmask = glow << gshift;
+    const int64_t s = a.seg_lo + ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+
+    int64_t e = 0, e_end = 0;
+    int rank = 0, slot_head = -1, slot_tail = -1;
+    if (s < a.seg_hi) {
+        const Segment g = a.segs[s];
+        e = g.start;
+        e_end = a.segs[s + 1].start;
+        rank = g.rank;
+        slot_head = g.slot_head;
+        slot_tail = g.slot_tail;
+    }
+    bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
+    bool open = false;                   // edges accumulated since the last store
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    while (__any_sync(kFull, e < e_end)) {
+        // ---- this chunk's edges: lane gl of the group owns edge e + gl
+        const int64_t left = e_end - e;
+        const int cnt = left >= G ? G : (left > 0 ? (int)left : 0);
+        uint32_t c = 0;
+        if (gl < cnt) c = a.colx[e + gl - a.colx_base];
+        const unsigned ends = (__ballot_sync(kFull, (c & kRowEndBit) != 0) >> gshift) & glow;
+        const int my_rank = rank + __popc(ends & ((1u << gl) - 1u));
+        const int col = (int)(c & ~kRowEndBit);
+        int my_row = my_rank;
+        float my_r = 1.f, w = 1.f;
+        if (c & kRowEndBit) {
+            if (HAS_EMPTY) my_row = a.nzrows[my_rank];
+            if (OP != GNNPRE_OP_GIN_SUM) my_r = a.rscale[my_row];
+        }
+        if (OP == GNNPRE_OP_GCN_SYM) {
+            if (gl < cnt) w = a.cscale[col];
+        } else if (OP == GNNPRE_OP_GIN_SUM) {
+            w = col == my_row ? a.diag_weight : 1.f;  // every row owns its self-loop, so rank == row
+        }
+        const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
+
+        // ---- gather and accumulate, U rows in flight
+        for (int t0 = 0; t0 < cnt_max; t0 += U) {
+            float4 x[U][V];
+            uint32_t craw[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int t = t0 + u;  // may run past G - 1 in the last step: the shuffle wraps, `ok` masks it
+                craw[u] = __shfl_sync(kFull, c, t & (G - 1), G);
+                const bool ok = t < cnt;
+                const float* row = a.x + (int64_t)(craw[u] & ~kRowEndBit) * a.ldx;
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const int q = gl + v * G;
+                    x[u][v] = (ok && q < a.f4) ? ld_row(row + 4 * q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int t = t0 + u;
+                const bool ok = t < cnt;
+                float ww = 1.f;
+                if (OP != GNNPRE_OP_SAGE_MEAN) ww = __shfl_sync(kFull, w, t & (G - 1), G);
+#pragma unroll
+                for (int v = 0; v < V; ++v) fma4(acc[v], ww, x[u][v]);
+                if (ok) open = true;
+                if (ok && (craw[u] & kRowEndBit)) {
+                    // last edge of a row: all lanes of the group arrive here together
+                    const int row = __shfl_sync(gmask, my_row, gshift + t);
+                    const float r = __shfl_sync(gmask, my_r, gshift + t);
+                    float* dst;
+                    float scale;
+                    if (head_pending) {  // the row began earlier: leave the partial sum for the fix-up
+                        dst = a.scratch + (int64_t)slot_head * a.scratch_ld;
+                        scale = 1.f;
+                        head_pending = false;
+                    } else {
+                        dst = a.out + (int64_t)row * a.ldo;
+                        scale = r;
+                    }
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        const int q = gl + v * G;
+                        if (q < a.f4) {
+                            float4 o = acc[v];
+                            o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
+                            *reinterpret_cast<float4*>(dst + 4 * q) = o;
+                        }
+                        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    open = false;
+                }
+            }
+        }
+        rank += __popc(ends);
+        e += G;
+    }
+
+    // ---- the row holding the last edge continues in the next segment
+    if (open) {
+        const int slot = head_pending ? slot_head : slot_tail;
+        if (slot >= 0) {
+            float* dst = a.scratch + (int64_t)slot * a.scratch_ld;
+#pragma unroll
+            for (int v = 0; v < V; ++v) {
+                const int q = gl + v * G;
+                if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = acc[v];
+            }
+        }
+    }
+}
+
+struct FixArgs {
+    const RowFixup* fix;
+    int64_t fix_lo, fix_hi;
+    const Segment* segs;
+    const float* scratch;
+    int64_t scratch_ld;
+    const float* rscale;
+    float* out;
+    int64_t ldo;
+    int32_t f4;
+};
+
+// One group per cut row: tail part of its first segment, then the head parts of the following ones,
+// added in segment order.
+template <int G, int V>
+__global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
+    constexpr unsigned kFull = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (G - 1);
+    const int64_t i = a.fix_lo + ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+    int first = 0, last = -1, row = 0;
+    if (i < a.fix_hi) {
+        const RowFixup f = a.fix[i];
+        first = f.seg_first;
+        last = f.seg_last;
+        row = f.row;
+    }
+    float4 acc[V];
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    int s0 = first;
+    while (__any_sync(kFull, s0 <= last)) {
+        const int cnt = last - s0 + 1 >= G ? G : (last >= s0 ? last - s0 + 1 : 0);
+        int slot = -1;
+        if (gl < cnt) {
+            const int s = s0 + gl;
+            slot = s == first ? a.segs[s].slot_tail : a.segs[s].slot_head;
+        }
+        const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
+        for (int t = 0; t < cnt_max; ++t) {
+            const int sl = __shfl_sync(kFull, slot, t, G);
+            if (t < cnt && sl >= 0) {
+                const float* p = a.scratch + (int64_t)sl * a.scratch_ld;
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    const int q = gl + v * G;
+                    if (q < a.f4) {
+                        const float4 x = *reinterpret_cast<const float4*>(p + 4 * q);
+                        acc[v].x += x.x; acc[v].y += x.y; acc[v].z += x.z; acc[v].w += x.w;
+                    }
+                }
+            }
+        }
+        s0 += G;
+    }
+    if (i < a.fix_hi) {
+        const float r = a.rscale[row];
+        float* dst = a.out + (int64_t)row * a.ldo;
+#pragma unroll
+        for (int v = 0; v < V; ++v) {
+            const int q = gl + v * G;
+            if (q < a.f4) {
+                float4 o = acc[v];
+                o.x *= r; o.y *= r; o.z *= r; o.w *= r;
+                *reinterpret_cast<float4*>(dst + 4 * q) = o;
+            }
+        }
+    }
+}
+
+// Rows without any edge (SAGE, D_i = 0) are zero rows of the result.
+__global__ void k_zero_rows(const int32_t* __restrict__ rows, int64_t count, float* __restrict__ out, int64_t ldo,
+                            int32_t f4) {
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= count * f4) return;
+    const int64_t r = rows[t / f4];
+    *reinterpret_cast<float4*>(out + r * ldo + 4 * (t % f4)) = make_float4(0.f, 0.f, 0.f, 0.f);
+}
+
+template <int G, int V, int U>
+int launch_segments_shape(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
+    const int64_t groups = a.seg_hi - a.seg_lo;
+    const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
+    switch (P->op) {
+    case GNNPRE_OP_GCN_SYM:
+        k_segments<G, V, U, GNNPRE_OP_GCN_SYM, false><<<grid, kThreads, 0, st>>>(a);
+        break;
+    case GNNPRE_OP_GIN_SUM:
+        k_segments<G, V, U, GNNPRE_OP_GIN_SUM, false><<<grid, kThreads, 0, st>>>(a);
+        break;
+    default:
+        if (P->rows_all_nonempty)
+            k_segments<G, V, U, GNNPRE_OP_SAGE_MEAN, false><<<grid, kThreads, 0, st>>>(a);
+        else
+            k_segments<G, V, U, GNNPRE_OP_SAGE_MEAN, true><<<grid, kThreads, 0, st>>>(a);
+    }
+    GNNPRE_CUDA(cudaGetLastError());
+    return GNNPRE_OK;
+}
+
+template <int G, int V>
+int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
+    const int64_t groups = a.fix_hi - a.fix_lo;
+    const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
+    k_row_fixups<G, V><<<grid, kThreads, 0, st>>>(a);
+    GNNPRE_CUDA(cudaGetLastError());
+    return GNNPRE_OK;
+}
+
+constexpr int kMaxTile = 512;  // columns one launch covers (G = 32, V = 4)
+
+}  // namespace
+
+int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int64_t seg_hi, cudaStream_t st) {
+    if (seg_hi <= seg_lo) return GNNPRE_OK;
+    for (int32_t f0 = 0; f0 < h.width; f0 += kMaxTile) {
+        const int32_t w = std::min<int32_t>(kMaxTile, h.width - f0);
+        SegArgs a;
+        a.segs = P->segments.p;
+        a.seg_lo = seg_lo;
+        a.seg_hi = seg_hi;
+        a.colx = h.colx;
+        a.colx_base = h.colx_edge_base;
+        a.x = h.xprev + f0;
+        a.ldx = h.ldx;
+        a.out = h.xout + f0;
+        a.ldo = h.ldo;
+        a.scratch = P->scratch.p + f0;
+        a.scratch_ld = P->slab_width;
+        a.rscale = P->rscale.p;
+        a.cscale = P->cscale.p;
+        a.nzrows = P->nzrows.p;
+        a.f4 = w / 4;
+        a.diag_weight = 1.0f + P->gin_eps;
+        if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
+        else if (a.f4 <= 8) GNNPRE_TRY((launch_segments_shape<8, 1, 8>(P, a, st)));
+        else if (a.f4 <= 16) GNNPRE_TRY((launch_segments_shape<16, 1, 8>(P, a, st)));
+        else if (a.f4 <= 32) GNNPRE_TRY((launch_segments_shape<32, 1, 8>(P, a, st)));
+        else if (a.f4 <= 64) GNNPRE_TRY((launch_segments_shape<32, 2, 4>(P, a, st)));
+        else GNNPRE_TRY((launch_segments_shape<32, 4, 2>(P, a, st)));
+    }
+    return GNNPRE_OK;
+}
+
+int launch_fixups(const gnnpre_plan* P, const HopArgs& h, int64_t fix_lo, int64_t fix_hi, cudaStream_t st) {
+    if (fix_hi <= fix_lo) return GNNPRE_OK;
+    for (int32_t f0 = 0; f0 < h.width; f0 += kMaxTile) {
+        const int32_t w = std::min<int32_t>(kMaxTile, h.width - f0);
+        FixArgs a;
+        a.fix = P->fixups.p;
+        a.fix_lo = fix_lo;
+        a.fix_hi = fix_hi;
+        a.segs = P->segments.p;
+        a.scratch = P->scratch.p + f0;
+        a.scratch_ld = P->slab_width;
+        a.rscale = P->rscale.p;
+        a.out = h.xout + f0;
+        a.ldo = h.ldo;
+        a.f4 = w / 4;
+        if (a.f4 <= 4) GNNPRE_TRY((launch_fixups_shape<4, 1>(a, st)));
+        else if (a.f4 <= 8) GNNPRE_TRY((launch_fixups_shape<8, 1>(a, st)));
+        else if (a.f4 <= 16) GNNPRE_TRY((launch_fixups_shape<16, 1>(a, st)));
+        else if (a.f4 <= 32) GNNPRE_TRY((launch_fixups_shape<32, 1>(a, st)));
+        else if (a.f4 <= 64) GNNPRE_TRY((launch_fixups_shape<32, 2>(a, st)));
+        else GNNPRE_TRY((launch_fixups_shape<32, 4>(a, st)));
+    }
+    return GNNPRE_OK;
+}
+
+int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t st) {
+    if (P->num_empty == 0) return GNNPRE_OK;
+    const int32_t f4 = h.width / 4;
+    const int64_t items = P->num_empty * f4;
+    k_zero_rows<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4);
+    GNNPRE_CUDA(cudaGetLastError());
+    return GNNPRE_OK;
+}
+
+// Everything on the device: K hops, each a sweep over the column slabs and the edge blocks.
+int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, float* const* out, int64_t ldo,
+                       cudaStream_t st, gnnpre_stats_t* stats) {
+    std::vector<cudaEvent_t> ev;
+    if (stats) {
+        ev.resize((size_t)K + 1);
+        for (auto& e : ev) GNNPRE_CUDA(cudaEventCreate(&e));
+        GNNPRE_CUDA(cudaEventRecord(ev[0], st));
+    }
+    int64_t launches = 0;
+    int rc = GNNPRE_OK;
+    for (int32_t k = 0; k < K && rc == GNNPRE_OK; ++k) {
+        const float* xprev = k == 0 ? X : out[k - 1];
+        const int64_t ldp = k == 0 ? ldx : ldo;
+        for (int32_t i = 0; i < P->c && rc == GNNPRE_OK; ++i) {
+            const int64_t f_lo = (int64_t)i * P->slab_width;
+            HopArgs h;
+            h.colx = P->colx.p;
+            h.colx_edge_base = 0;
+            h.xprev = xprev + f_lo;
+            h.ldx = ldp;
+            h.xout = out[k] + f_lo;
+            h.ldo = ldo;
+            h.width = (int32_t)std::min<int64_t>(P->slab_width, P->feat_dim - f_lo);
+            const int tiles = (h.width + kMaxTile - 1) / kMaxTile;
+            rc = launch_zero_empty_rows(P, h, st);
+            launches += P->num_empty ? 1 : 0;
+            if (rc != GNNPRE_OK) break;
+            if (P->flags & GNNPRE_FLAG_LAUNCH_PER_BLOCK) {
+                for (const Block& B : P->blocks) {
+                    rc = launch_segments(P, h, B.seg_lo, B.seg_hi, st);
+                    if (rc == GNNPRE_OK) rc = launch_fixups(P, h, B.fix_lo, B.fix_hi, st);
+                    if (rc != GNNPRE_OK) break;
+                    launches += tiles * ((B.seg_hi > B.seg_lo) + (B.fix_hi > B.fix_lo));
+                }
+            } else {
+                rc = launch_segments(P, h, 0, P->num_segments, st);
+                if (rc == GNNPRE_OK) rc = launch_fixups(P, h, 0, P->num_fixups, st);
+                launches += tiles * ((P->num_segments > 0) + (P->num_fixups > 0));
+            }
+        }
+        if (stats && rc == GNNPRE_OK) {
+            cudaError_t e = cudaEventRecord(ev[(size_t)k + 1], st);
+            if (e != cudaSuccess) rc = GNNPRE_ERR_CUDA;
+        }
+    }
+    if (stats) {
+        if (rc == GNNPRE_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = GNNPRE_ERR_CUDA;
+        if (rc == GNNPRE_OK) {
+            for (int32_t k = 0; k < K; ++k) cudaEventElapsedTime(&stats->hop_ms[k], ev[(size_t)k], ev[(size_t)k + 1]);
+            cudaEventElapsedTime(&stats->total_ms, ev[0], ev[(size_t)K]);
+            stats->kernel_launches = launches;
+            stats->h2d_bytes = 0;
+            stats->d2h_bytes = 0;
+        }
+        for (auto& e : ev) cudaEventDestroy(e);
+    }
+    return rc;
+}
+
+}  // namespace gnnpre

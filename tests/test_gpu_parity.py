@@ -1,0 +1,261 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the fp64 CPU oracle.
+
+Integer outputs (degrees, the support's edge list, block tables, Eq. 12) must match bit for bit;
+scale factors are fp64-computed and rounded once, so they match bit for bit too; propagated
+features must stay within 1e-5 relative error per hop.
+"""
+import itertools
+
+import numpy as np
+import pytest
+import torch
+
+import gnnpre_inputs as gi
+import oracle as orc
+from parity_util import TOL, backward_error, check_all_hops, hop_error, to_np
+
+pytestmark = pytest.mark.gpu
+
+OPS = (0, 1, 2)
+EPS = 0.1
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2207_12000_b200 import binding
+    return binding
+
+
+def dev(g):
+    return g.rowptr.cuda(), g.colidx.cuda()
+
+
+def small_graphs():
+    yield "er33", gi.erdos_renyi(33, 70, 5)
+    yield "er1000", gi.erdos_renyi(1000, 6000, 6)
+    yield "rmat3000", gi.rmat(3000, 20000, 7, directed_candidates=True)
+    yield "star", gi.from_edge_list(700, [(0, j) for j in range(1, 650)])  # hub + isolated tail nodes
+    yield "path2", gi.from_edge_list(2, [(0, 1)])
+    yield "lonely", gi.from_edge_list(5, [])  # no edges at all
+
+
+# ------------------------------------------------------------------ plan parity (bit-exact)
+
+@pytest.mark.parametrize("name,g", list(small_graphs()) + [("c1", None)])
+@pytest.mark.parametrize("op", OPS)
+def test_plan_matches_oracle_bit_for_bit(B, name, g, op):
+    if g is None:
+        g = gi.make_graph(gi.WORKLOADS["c1"])
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    deg = orc.degrees(rp)
+    np.testing.assert_array_equal(to_np(B.gnnpre_degrees(drp, dci)), deg)
+    rp_t, ci_t = orc.support(op, rp, ci)
+    m = int(rp_t[-1])
+    for b in sorted({1, 2, 3, 7, 64, m} - {0}):
+        if b > m:
+            continue
+        plan = B.gnnpre_build_plan(drp, dci, op, 16, gin_eps=EPS, force_blocks=b, force_col_slabs=1, segment_edges=8)
+        info = plan.info()
+        assert (info["n"], info["nnz"], info["nnz_tilde"], info["b"], info["c"]) == (g.n, g.nnz, m, b, 1)
+        assert info["B_S"] == 4 * m + 8 * (g.n + 1) and info["B_X"] == 4 * g.n * 16
+        pdeg, r, c = B.gnnpre_plan_scales(plan)
+        np.testing.assert_array_equal(pdeg.numpy(), deg)
+        wr, wc = orc.scales_f32(op, deg)
+        np.testing.assert_array_equal(r.numpy().view(np.uint32), wr.view(np.uint32))
+        np.testing.assert_array_equal(c.numpy().view(np.uint32), wc.view(np.uint32))
+        srp, sci = B.gnnpre_plan_support(plan)
+        np.testing.assert_array_equal(srp.numpy(), rp_t)
+        np.testing.assert_array_equal(sci.numpy(), ci_t)
+        e_off = orc.block_offsets(m, b)
+        row_lo, row_hi, fp, lp = orc.block_rows(rp_t, e_off)
+        for l in range(b):
+            blk = B.gnnpre_plan_block(plan, l)
+            assert (blk["e_lo"], blk["e_hi"]) == (e_off[l], e_off[l + 1])
+            assert (blk["row_lo"], blk["row_hi"]) == (row_lo[l], row_hi[l])
+            assert (blk["first_row_partial"], blk["last_row_partial"]) == (fp[l], lp[l])
+        plan.close()
+
+
+def test_plan_with_caller_degrees_and_budget_search(B):
+    g = gi.erdos_renyi(500, 3000, 8)
+    drp, dci = dev(g)
+    deg = B.gnnpre_degrees(drp, dci)
+    F = 64
+    m = g.nnz + g.n
+    B_S, B_X, B_fixed = 4 * m + 8 * (g.n + 1), 4 * g.n * F, 16 * g.n
+    for budget in (B_fixed + B_S + 2 * B_X, B_fixed + B_S // 3 + B_X, B_fixed + 2000 + B_X // 2):
+        want = orc.solve_budget(B_S, B_X, B_fixed, 1, 2, budget, min(m, 1 << 20), F // 4)
+        plan = B.gnnpre_build_plan(drp, dci, 0, F, degrees=deg, budget_bytes=budget)
+        info = plan.info()
+        assert (info["b"], info["c"]) == want
+        assert info["slab_width"] == orc.slab_width(F, info["c"])
+        plan.close()
+    with pytest.raises(B.GnnpreError) as ei:
+        B.gnnpre_build_plan(drp, dci, 0, F, budget_bytes=B_fixed + 100)
+    assert ei.value.status == -6
+
+
+# ------------------------------------------------------------------ propagation parity
+
+def run_case(B, g, op, F, K, *, b=1, c=1, seg=0, flags=0, ldx=None, ldo=None, seed=1):
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    ldx = ldx or F
+    ldo = ldo or F
+    Xbuf = torch.full((g.n, ldx), float("nan"), device="cuda")
+    X = Xbuf[:, :F]
+    X.copy_(gi.normal_matrix(g.n, F, seed, device="cuda"))
+    obufs = [torch.full((g.n, ldo), -7.0, device="cuda") for _ in range(K)]
+    outs = [o[:, :F] for o in obufs]
+    plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c, segment_edges=seg,
+                               flags=flags)
+    B.gnnpre_propagate(plan, X, K, outs)
+    torch.cuda.synchronize()
+    for o in obufs:
+        assert bool((o[:, F:] == -7.0).all()), "padding columns were written"
+    worst = check_all_hops(op, EPS, rp, ci, to_np(X), outs)
+    plan.close()
+    return worst, outs
+
+
+def test_config1_erdos_renyi_gcn(B):
+    """Configuration 1: 4,096 nodes, 32,768 edges, F=64, K=2, GCN, a single edge block."""
+    w = gi.WORKLOADS["c1"]
+    g = gi.make_graph(w)
+    assert (g.n, g.nnz) == (4096, 65536)
+    run_case(B, g, w.op, w.feat_dim, w.hops, b=w.blocks, seed=w.seed)
+
+
+@pytest.mark.parametrize("name,g", list(small_graphs()))
+@pytest.mark.parametrize("op", OPS)
+def test_small_graphs_all_shapes(B, name, g, op):
+    m = orc.support_nnz(op, g.n, g.nnz)
+    for F, seg in ((4, 8), (16, 4), (20, 32), (64, 8), (100, 16), (128, 0), (256, 8), (516, 32), (1040, 8)):
+        for b in (1, 3):
+            if b > m:
+                continue
+            run_case(B, g, op, F, 2, b=b, seg=seg)
+
+
+@pytest.mark.parametrize("op", OPS)
+def test_blocks_slabs_and_launch_modes_agree(B, op):
+    """Different (b, c), segment sizes and launch groupings change only the rounding order."""
+    g = gi.rmat(5000, 40000, 9, directed_candidates=True)
+    F, K = 72, 3
+    ref = None
+    for b, c, seg, flags in ((1, 1, 0, 0), (4, 1, 64, 0), (64, 1, 16, 1), (7, 3, 32, 1), (1, 18, 1, 0), (5, 2, 0, 0)):
+        _, outs = run_case(B, g, op, F, K, b=b, c=c, seg=seg, flags=flags, ldx=F + 4, ldo=F + 8)
+        cur = [to_np(o).astype(np.float64) for o in outs]
+        if ref is None:
+            ref = cur
+        else:
+            for k in range(K):
+                assert hop_error(cur[k], ref[k]) <= TOL
+
+
+def test_hub_longer_than_many_segments_and_blocks(B):
+    """A row far longer than a segment and a block: its parts are summed by the fix-up pass."""
+    n = 40000
+    edges = [(0, j) for j in range(1, n)] + [(j, j + 1) for j in range(1, 2000)]
+    g = gi.from_edge_list(n, edges)
+    for op in OPS:
+        run_case(B, g, op, 32, 2, b=9, seg=32)
+        run_case(B, g, op, 128, 2, b=1, seg=0)
+
+
+def test_runs_are_bitwise_reproducible(B):
+    g = gi.rmat(20000, 200000, 10, directed_candidates=True)
+    drp, dci = dev(g)
+    X = gi.normal_matrix(g.n, 128, 3, device="cuda")
+    plan = B.gnnpre_build_plan(drp, dci, 0, 128, force_blocks=4)
+    a, _ = B.gnnpre_propagate(plan, X, 3)
+    b, _ = B.gnnpre_propagate(plan, X, 3)
+    torch.cuda.synchronize()
+    for x, y in zip(a, b):
+        assert torch.equal(x, y)
+    plan.close()
+
+
+def test_config2_rmat_gcn_four_blocks(B):
+    """Configuration 2: 169,343 nodes, 1,166,243 directed R-MAT edges symmetrised, F=128, K=3, GCN, b=4."""
+    w = gi.WORKLOADS["c2"]
+    g = gi.make_graph(w, device="cuda").to("cpu")
+    assert g.n == 169343
+    run_case(B, g, w.op, w.feat_dim, w.hops, b=w.blocks, seed=w.seed)
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("F", [16, 64, 128, 256, 512])
+def test_config3_operator_width_block_sweep(B, op, F):
+    """Configuration 3: ops x widths x block counts {1, 8, 64} on the 169,343-node graph, K=3."""
+    w = gi.WORKLOADS["c3"]
+    g = gi.make_graph(w, device="cuda").to("cpu")
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    X = gi.normal_matrix(g.n, F, w.seed, device="cuda")
+    Xn = to_np(X)
+    want = orc.propagate(op, w.gin_eps, rp, ci, Xn, w.hops)
+    for b in w.sweep["blocks"]:
+        plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=w.gin_eps, force_blocks=b)
+        outs, _ = B.gnnpre_propagate(plan, X, w.hops)
+        torch.cuda.synchronize()
+        prev = Xn
+        for k in range(w.hops):
+            gk = to_np(outs[k])
+            assert hop_error(gk, want[k]) <= TOL
+            rows = np.random.default_rng(k).integers(0, g.n, 4096)
+            assert backward_error(op, w.gin_eps, rp, ci, prev, gk, rows) <= TOL
+            prev = gk
+        plan.close()
+
+
+# ------------------------------------------------------------------ errors and edge cases
+
+def test_invalid_inputs_are_rejected(B):
+    g = gi.erdos_renyi(100, 300, 11)
+    drp, dci = dev(g)
+
+    def status(fn):
+        with pytest.raises(B.GnnpreError) as ei:
+            fn()
+        return ei.value.status
+
+    assert status(lambda: B.gnnpre_build_plan(drp, dci, 0, 18)) == -3          # F % 4
+    assert status(lambda: B.gnnpre_build_plan(drp, dci, 5, 16)) == -1          # bad op
+    assert status(lambda: B.gnnpre_build_plan(drp, dci, 1, 16, force_blocks=g.nnz + 1)) == -1  # empty block
+    assert status(lambda: B.gnnpre_build_plan(drp, dci, 0, 16, force_col_slabs=5)) == -1
+    bad = dci.clone()
+    bad[3] = 10 ** 6
+    assert status(lambda: B.gnnpre_build_plan(drp, bad, 0, 16)) == -2          # column out of range
+    bad = dci.clone()
+    bad[int(g.rowptr[5])] = 5
+    assert status(lambda: B.gnnpre_build_plan(drp, bad, 0, 16)) == -2          # a diagonal entry or broken order
+    bad = dci.clone()
+    lo = int(g.rowptr[7])
+    bad[lo + 1] = bad[lo]
+    assert status(lambda: B.gnnpre_build_plan(drp, bad, 0, 16)) == -2          # duplicate column
+    badrp = drp.clone()
+    badrp[10] = badrp[11] + 1
+    assert status(lambda: B.gnnpre_build_plan(badrp, dci, 0, 16)) == -2        # rowptr not monotone
+    plan = B.gnnpre_build_plan(drp, dci, 0, 16)
+    X = torch.zeros((100, 18), device="cuda")[:, :16]
+    assert status(lambda: B.gnnpre_propagate(plan, X, 1)) == -3               # ldx % 4
+    X = torch.zeros((100, 16), device="cuda")
+    assert status(lambda: B.gnnpre_propagate(plan, X, 0, [])) == -1
+    assert status(lambda: B.gnnpre_propagate(plan, X, 2, [X.clone(), X])) == -1  # out aliases X
+    plan.close()
+
+
+def test_graph_without_edges(B):
+    g = gi.from_edge_list(6, [])
+    drp, dci = dev(g)
+    X = gi.normal_matrix(6, 8, 1, device="cuda")
+    for op, want in ((0, X), (1, torch.zeros_like(X)), (2, (1 + np.float32(EPS)) * X)):
+        plan = B.gnnpre_build_plan(drp, dci, op, 8, gin_eps=EPS)
+        outs, _ = B.gnnpre_propagate(plan, X, 2)
+        torch.cuda.synchronize()
+        torch.testing.assert_close(outs[0], want, rtol=1e-6, atol=0)
+        plan.close()
