@@ -1,0 +1,309 @@
+#!/usr/bin/env python
+"""Benchmark of block-wise multi-hop feature aggregation on B200.
+
+A step is one gnnpre_propagate call: all K hops over every edge block of one synthetic workload.
+The metric is propagated edge-feature elements per second, K * |E| * F / t, where |E| counts the
+edges of the operator's support.  One JSON line is printed by rank 0.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4] [--impl ours|reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs an independent replica of the same
+workload on its own GPU; the path has no exchange step, so there is no collective in it.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+import gnnpre_inputs as gi
+
+METRIC = "propagated edge-feature elems/s over K hops"
+UNIT = "elems/s"
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c4", choices=sorted(gi.WORKLOADS))
+    ap.add_argument("--scale-down", type=int, default=1, help="divide nodes and edges (debugging only)")
+    ap.add_argument("--segment-edges", type=int, default=0)
+    ap.add_argument("--blocks", type=int, default=-1, help="override the workload's block count")
+    ap.add_argument("--per-block-launch", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                      "-i", str(self.index)], capture_output=True, text=True, timeout=5).stdout
+                parts = [p.strip() for p in out.strip().split(",")]
+                if len(parts) == 6:
+                    self.rows.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.1)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        if not self.rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unsampled"]}
+        sm = sorted(float(r[0]) for r in self.rows)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[2 + i] == "Active" for r in self.rows)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.rows[0][1]), "reasons": reasons,
+                "samples": len(self.rows)}
+
+
+def byte_model(n, m, F):
+    """Algorithmic bytes of one hop.  gather: every neighbour row comes from memory once per edge;
+    min: every matrix is touched once."""
+    gather = 4 * m * F + 4 * n * F + 4 * m + 16 * n
+    least = 8 * n * F + 4 * m + 16 * n
+    return gather, least
+
+
+def oracle_sample(w, g_cpu, X_cpu, target_seconds):
+    """Times the CPU oracle, as it stands, on a row range of hop 1 sized for about target_seconds."""
+    import oracle as orc
+    rp, ci = g_cpu.rowptr.numpy(), g_cpu.colidx.numpy()
+    n = g_cpu.n
+    diag = 0 if w.op == gi.OP_SAGE else 1
+    probe_rows = max(1, n // 256)
+    t0 = time.perf_counter()
+    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(probe_rows), want_abs=False)
+    t_probe = time.perf_counter() - t0
+    probe_edges = int(rp[probe_rows]) + diag * probe_rows
+    rate = probe_edges / max(t_probe, 1e-6)
+    want_edges = rate * target_seconds
+    total_edges = int(rp[n]) + diag * n
+    rows = n if want_edges >= total_edges else int(np.searchsorted(rp, want_edges))
+    rows = max(1, min(n, rows))
+    t0 = time.perf_counter()
+    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(rows), want_abs=False)
+    t = time.perf_counter() - t0
+    edges = int(rp[rows]) + diag * rows
+    return {"value": edges * X_cpu.shape[1] / t, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+            "sample": f"hop 1 of {w.name} on rows [0, {rows}) = {edges} of {total_edges} edges, {t:.2f} s"}, t
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: every step is a bounded sample of the workload on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    g = gi.make_graph(w, device=dev).to("cpu")
+    X = gi.make_features(w, device=dev).cpu().numpy()
+    per_step = min(args.cpu_seconds, 120.0 / max(1, args.steps + args.warmup))
+    vals, ms = [], []
+    base = None
+    for i in range(args.warmup + args.steps):
+        base, t = oracle_sample(w, g, X, per_step)
+        if i >= args.warmup:
+            vals.append(base["value"])
+            ms.append(t * 1e3)
+    value = float(np.mean(vals))
+    base["value"] = value
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": float(np.mean(ms)), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": workload_config(w, g, None), "cpu_baseline": base,
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(w, g, info):
+    cfg = {"workload": f"{w.name}: {w.kind} graph, {g.n} nodes, {g.nnz} directed nnz, F={w.feat_dim}, K={w.hops}, "
+                       f"op={('gcn_sym', 'sage_mean', 'gin_sum')[w.op]}",
+           "l2_policy": "inputs larger than L2 (X and every hop are n*F*4 bytes each; no flush between steps)"
+           if g.n * w.feat_dim * 4 > 126e6 else "L2 flushed between steps by writing a 256 MB buffer"}
+    if info:
+        cfg.update({"blocks": info["b"], "col_slabs": info["c"], "segment_edges": info["segment_edges"],
+                    "nnz_tilde": info["nnz_tilde"]})
+    return cfg
+
+
+def main():
+    args = parse()
+    w = gi.scaled(gi.WORKLOADS[args.workload], args.scale_down)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    from paper_2207_12000_b200 import binding as B  # fails loudly if the CUDA library is missing
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---------------- inputs (seeded, generated on the device, resident before timing starts)
+    t0 = time.perf_counter()
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    torch.cuda.synchronize()
+    gen_s = time.perf_counter() - t0
+    K, F = w.hops, w.feat_dim
+    blocks = w.blocks if args.blocks < 0 else args.blocks
+    flags = B.GNNPRE_FLAG_LAUNCH_PER_BLOCK if args.per_block_launch else 0
+
+    t0 = time.perf_counter()
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
+                               force_col_slabs=1 if blocks else 0, segment_edges=args.segment_edges, flags=flags)
+    torch.cuda.synchronize()
+    plan_ms = (time.perf_counter() - t0) * 1e3
+    info = plan.info()
+    m = info["nnz_tilde"]
+    outs = [torch.empty((g.n, F), dtype=torch.float32, device="cuda") for _ in range(K)]
+    small = g.n * F * 4 <= 126e6
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
+    stream = torch.cuda.current_stream()
+
+    def step(want_stats):
+        if flush is not None:
+            flush.fill_(1)
+        _, st = B.gnnpre_propagate(plan, X, K, outs, stream=stream, want_stats=want_stats)
+        return st
+
+    for _ in range(max(3, args.warmup)):
+        step(False)
+    barrier()
+
+    # ---------------- timed region: device-resident inputs, CUDA events on the launching stream
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    seg_ms, seg_launches, launches = 0.0, 0, 0
+    with ClockSampler(local) as clocks:
+        barrier()
+        for a, b_ in ev:
+            a.record(stream)
+            st = step(True)
+            b_.record(stream)
+            seg_ms += st.segments_ms
+            seg_launches += st.segments_launches
+            launches += st.kernel_launches
+        barrier()
+    step_ms = [a.elapsed_time(b_) for a, b_ in ev]
+    total_ms = float(sum(step_ms))
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    units_per_step = K * m * F
+    value = world * units_per_step * args.steps / (total_ms * 1e-3)
+
+    # ---------------- roofline of the dominant kernel (the segment kernel: one launch = one hop here)
+    peak, peak_kind = measured_peaks()
+    gather_b, least_b = byte_model(g.n, m, F)
+    launches_per_hop = seg_launches / (args.steps * K)
+    seg_launch_ms = seg_ms / max(1, seg_launches)
+    achieved = gather_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": None,
+                "kernel": "k_segments", "kernel_ms_per_launch": seg_launch_ms,
+                "algorithmic_bytes_per_launch": gather_b / launches_per_hop,
+                "achieved_min_model": least_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9,
+                "kernel_share_of_step": seg_ms / total_ms if world == 1 else None}
+
+    # ---------------- end to end through the C ABI with host buffers (copies inside the timed region)
+    e2e = None
+    if not args.no_e2e and rank == 0:
+        try:
+            Xh = torch.empty((g.n, F), dtype=torch.float32, pin_memory=True)
+            Xh.copy_(X)
+            outs_h = [torch.empty((g.n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
+            hplan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
+                                        force_col_slabs=0, segment_edges=args.segment_edges,
+                                        operands_mem=B.GNNPRE_MEM_HOST)
+            for _ in range(2):
+                B.gnnpre_propagate(hplan, Xh, K, outs_h)
+            reps = max(2, min(args.steps, 5))
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            for _ in range(reps):
+                _, hst = B.gnnpre_propagate(hplan, Xh, K, outs_h, want_stats=True)
+            torch.cuda.synchronize()
+            dt = (time.perf_counter() - t0) / reps
+            e2e = {"value": units_per_step / dt, "unit": UNIT, "h2d_bytes_per_step": int(hst.h2d_bytes),
+                   "d2h_bytes_per_step": int(hst.d2h_bytes), "ms_per_step": dt * 1e3,
+                   "col_slabs": hplan.info()["c"]}
+            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if hplan.info()["c"] == 1 else None
+            e2e["bitwise_equal_to_resident"] = same
+            hplan.close()
+        except B.GnnpreError as err:
+            e2e = {"value": None, "unit": UNIT, "error": str(err)}
+
+    # ---------------- the oracle on this machine's host cores, bounded sample (rank 0, one GPU only)
+    cpu = None
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        cpu, _ = oracle_sample(w, g.to("cpu"), X.cpu().numpy(), args.cpu_seconds)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": workload_config(w, g, info), "clocks": clocks.summary(), "e2e": e2e,
+                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
+                "plan_build_ms": plan_ms, "input_generation_s": gen_s,
+                "hop_ms": [float(st.hop_ms[k]) for k in range(K)]}
+        print(json.dumps(line), flush=True)
+    plan.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

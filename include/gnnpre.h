@@ -114,8 +114,10 @@ typedef struct {
 typedef struct {
     float hop_ms[GNNPRE_MAX_HOPS]; /* device time per hop (CUDA events); device-resident runs with stats only */
     float total_ms;
+    float segments_ms;             /* device time spent in the segment kernel alone, summed over its launches */
     int64_t h2d_bytes, d2h_bytes;  /* streamed runs */
-    int64_t kernel_launches;
+    int64_t kernel_launches;       /* all kernels this call launched */
+    int64_t segments_launches;     /* launches of the segment kernel among them */
 } gnnpre_stats_t;
 
 /*

@@ -54,7 +54,8 @@ class gnnpre_block_info_t(ctypes.Structure):
 
 class gnnpre_stats_t(ctypes.Structure):
     _fields_ = [("hop_ms", ctypes.c_float * GNNPRE_MAX_HOPS), ("total_ms", ctypes.c_float),
-                ("h2d_bytes", ctypes.c_int64), ("d2h_bytes", ctypes.c_int64), ("kernel_launches", ctypes.c_int64)]
+                ("segments_ms", ctypes.c_float), ("h2d_bytes", ctypes.c_int64), ("d2h_bytes", ctypes.c_int64),
+                ("kernel_launches", ctypes.c_int64), ("segments_launches", ctypes.c_int64)]
 
 
 class GnnpreError(RuntimeError):

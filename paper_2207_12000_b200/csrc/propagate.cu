@@ -45,6 +45,23 @@ __device__ __forceinline__ void fma4(float4& a, float w, const float4& x) {
     a.w = fmaf(w, x.w, a.w);
 }
 
+// Compensated (Kahan) addition of x into the pair (sum, comp).  The sums over the edges of one chunk
+// are short and plain; the long chains (chunk sums of a segment, segment parts of a cut row) are
+// compensated, so the error of a row's sum does not grow with its degree.
+__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) {
+    const float y = x - comp;
+    const float t = sum + y;
+    comp = (t - sum) - y;
+    sum = t;
+}
+
+__device__ __forceinline__ void kahan4(float4& sum, float4& comp, const float4& x) {
+    kahan1(sum.x, comp.x, x.x);
+    kahan1(sum.y, comp.y, x.y);
+    kahan1(sum.z, comp.z, x.z);
+    kahan1(sum.w, comp.w, x.w);
+}
+
 constexpr int kThreads = 256;
 
 // G lanes per segment, V float4 per lane (row width <= 4*G*V floats), U rows in flight per lane.
@@ -70,9 +87,9 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
     }
     bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
     bool open = false;                   // edges accumulated since the last store
-    float4 acc[V];
+    float4 acc[V], tot[V], cmp[V];       // this chunk's sum; the row's running sum and its compensation
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
     while (__any_sync(kFull, e < e_end)) {
         // ---- this chunk's edges: lane gl of the group owns edge e + gl
@@ -138,16 +155,22 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         const int q = gl + v * G;
+                        kahan4(tot[v], cmp[v], acc[v]);
                         if (q < a.f4) {
-                            float4 o = acc[v];
+                            float4 o = tot[v];
                             o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
                             *reinterpret_cast<float4*>(dst + 4 * q) = o;
                         }
-                        acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                     open = false;
                 }
             }
+        }
+#pragma unroll
+        for (int v = 0; v < V; ++v) {  // fold the chunk into the row's running sum
+            kahan4(tot[v], cmp[v], acc[v]);
+            acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         rank += __popc(ends);
         e += G;
@@ -161,7 +184,7 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
 #pragma unroll
             for (int v = 0; v < V; ++v) {
                 const int q = gl + v * G;
-                if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = acc[v];
+                if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = tot[v];
             }
         }
     }
@@ -194,9 +217,9 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
         last = f.seg_last;
         row = f.row;
     }
-    float4 acc[V];
+    float4 acc[V], cmp[V];
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) acc[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
     int s0 = first;
     while (__any_sync(kFull, s0 <= last)) {
         const int cnt = last - s0 + 1 >= G ? G : (last >= s0 ? last - s0 + 1 : 0);
@@ -214,8 +237,7 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
                 for (int v = 0; v < V; ++v) {
                     const int q = gl + v * G;
                     if (q < a.f4) {
-                        const float4 x = *reinterpret_cast<const float4*>(p + 4 * q);
-                        acc[v].x += x.x; acc[v].y += x.y; acc[v].z += x.z; acc[v].w += x.w;
+                        kahan4(acc[v], cmp[v], *reinterpret_cast<const float4*>(p + 4 * q));
                     }
                 }
             }
@@ -348,14 +370,18 @@ int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t 
 // Everything on the device: K hops, each a sweep over the column slabs and the edge blocks.
 int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, float* const* out, int64_t ldo,
                        cudaStream_t st, gnnpre_stats_t* stats) {
-    std::vector<cudaEvent_t> ev;
-    if (stats) {
-        ev.resize((size_t)K + 1);
-        for (auto& e : ev) GNNPRE_CUDA(cudaEventCreate(&e));
-        GNNPRE_CUDA(cudaEventRecord(ev[0], st));
-    }
-    int64_t launches = 0;
-    int rc = GNNPRE_OK;
+    // With stats, events bracket every hop and every launch of the segment kernel.
+    std::vector<cudaEvent_t> hop_ev, seg_ev;
+    auto mark = [&](std::vector<cudaEvent_t>& v) -> int {
+        if (!stats) return GNNPRE_OK;
+        cudaEvent_t e;
+        GNNPRE_CUDA(cudaEventCreate(&e));
+        v.push_back(e);
+        GNNPRE_CUDA(cudaEventRecord(e, st));
+        return GNNPRE_OK;
+    };
+    int64_t launches = 0, seg_launches = 0;
+    int rc = mark(hop_ev);
     for (int32_t k = 0; k < K && rc == GNNPRE_OK; ++k) {
         const float* xprev = k == 0 ? X : out[k - 1];
         const int64_t ldp = k == 0 ? ldx : ldo;
@@ -372,35 +398,47 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
             const int tiles = (h.width + kMaxTile - 1) / kMaxTile;
             rc = launch_zero_empty_rows(P, h, st);
             launches += P->num_empty ? 1 : 0;
-            if (rc != GNNPRE_OK) break;
-            if (P->flags & GNNPRE_FLAG_LAUNCH_PER_BLOCK) {
-                for (const Block& B : P->blocks) {
-                    rc = launch_segments(P, h, B.seg_lo, B.seg_hi, st);
-                    if (rc == GNNPRE_OK) rc = launch_fixups(P, h, B.fix_lo, B.fix_hi, st);
-                    if (rc != GNNPRE_OK) break;
-                    launches += tiles * ((B.seg_hi > B.seg_lo) + (B.fix_hi > B.fix_lo));
+            const bool per_block = (P->flags & GNNPRE_FLAG_LAUNCH_PER_BLOCK) != 0;
+            const size_t groups = per_block ? P->blocks.size() : 1;
+            for (size_t j = 0; j < groups && rc == GNNPRE_OK; ++j) {
+                const int64_t seg_lo = per_block ? P->blocks[j].seg_lo : 0;
+                const int64_t seg_hi = per_block ? P->blocks[j].seg_hi : P->num_segments;
+                const int64_t fix_lo = per_block ? P->blocks[j].fix_lo : 0;
+                const int64_t fix_hi = per_block ? P->blocks[j].fix_hi : P->num_fixups;
+                if (seg_hi > seg_lo) {
+                    rc = mark(seg_ev);
+                    if (rc == GNNPRE_OK) rc = launch_segments(P, h, seg_lo, seg_hi, st);
+                    if (rc == GNNPRE_OK) rc = mark(seg_ev);
+                    launches += tiles;
+                    seg_launches += tiles;
                 }
-            } else {
-                rc = launch_segments(P, h, 0, P->num_segments, st);
-                if (rc == GNNPRE_OK) rc = launch_fixups(P, h, 0, P->num_fixups, st);
-                launches += tiles * ((P->num_segments > 0) + (P->num_fixups > 0));
+                if (rc == GNNPRE_OK && fix_hi > fix_lo) {
+                    rc = launch_fixups(P, h, fix_lo, fix_hi, st);
+                    launches += tiles;
+                }
             }
         }
-        if (stats && rc == GNNPRE_OK) {
-            cudaError_t e = cudaEventRecord(ev[(size_t)k + 1], st);
-            if (e != cudaSuccess) rc = GNNPRE_ERR_CUDA;
-        }
+        if (rc == GNNPRE_OK) rc = mark(hop_ev);
     }
     if (stats) {
         if (rc == GNNPRE_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = GNNPRE_ERR_CUDA;
         if (rc == GNNPRE_OK) {
-            for (int32_t k = 0; k < K; ++k) cudaEventElapsedTime(&stats->hop_ms[k], ev[(size_t)k], ev[(size_t)k + 1]);
-            cudaEventElapsedTime(&stats->total_ms, ev[0], ev[(size_t)K]);
+            for (int32_t k = 0; k < K; ++k) cudaEventElapsedTime(&stats->hop_ms[k], hop_ev[(size_t)k], hop_ev[(size_t)k + 1]);
+            cudaEventElapsedTime(&stats->total_ms, hop_ev[0], hop_ev[(size_t)K]);
+            float seg_ms = 0.f;
+            for (size_t j = 0; j + 1 < seg_ev.size(); j += 2) {
+                float ms = 0.f;
+                cudaEventElapsedTime(&ms, seg_ev[j], seg_ev[j + 1]);
+                seg_ms += ms;
+            }
+            stats->segments_ms = seg_ms;
             stats->kernel_launches = launches;
+            stats->segments_launches = seg_launches;
             stats->h2d_bytes = 0;
             stats->d2h_bytes = 0;
         }
-        for (auto& e : ev) cudaEventDestroy(e);
+        for (auto& e : hop_ev) cudaEventDestroy(e);
+        for (auto& e : seg_ev) cudaEventDestroy(e);
     }
     return rc;
 }
