@@ -38,22 +38,24 @@ struct SegArgs {
 
 __device__ __forceinline__ float4 ld_row(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
 
-__device__ __forceinline__ void fma4(float4& a, float w, const float4& x) {
-    a.x = fmaf(w, x.x, a.x);
-    a.y = fmaf(w, x.y, a.y);
-    a.z = fmaf(w, x.z, a.z);
-    a.w = fmaf(w, x.w, a.w);
-}
-
-// Compensated (Kahan) addition of x into the pair (sum, comp).  The sums over the edges of one chunk
-// are short and plain; the long chains (chunk sums of a segment, segment parts of a cut row) are
-// compensated, so the error of a row's sum does not grow with its degree.
-__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) {
-    const float y = x - comp;
+// Compensated (Kahan) summation in fp32: the pair (sum, comp) absorbs w*x with the low-order bits
+// that the addition drops carried in comp, so the error of a row's sum stays at a few ulps of
+// sum_j |w_j x_j| whatever the degree.  The kernel is bound by memory, not by these extra adds.
+__device__ __forceinline__ void kahan_fma1(float& sum, float& comp, float w, float x) {
+    const float y = fmaf(w, x, -comp);
     const float t = sum + y;
     comp = (t - sum) - y;
     sum = t;
 }
+
+__device__ __forceinline__ void kahan_fma4(float4& sum, float4& comp, float w, const float4& x) {
+    kahan_fma1(sum.x, comp.x, w, x.x);
+    kahan_fma1(sum.y, comp.y, w, x.y);
+    kahan_fma1(sum.z, comp.z, w, x.z);
+    kahan_fma1(sum.w, comp.w, w, x.w);
+}
+
+__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) { kahan_fma1(sum, comp, 1.f, x); }
 
 __device__ __forceinline__ void kahan4(float4& sum, float4& comp, const float4& x) {
     kahan1(sum.x, comp.x, x.x);
@@ -87,9 +89,9 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
     }
     bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
     bool open = false;                   // edges accumulated since the last store
-    float4 acc[V], tot[V], cmp[V];       // this chunk's sum; the row's running sum and its compensation
+    float4 tot[V], cmp[V];               // the row's running sum and its compensation
 #pragma unroll
-    for (int v = 0; v < V; ++v) acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
     while (__any_sync(kFull, e < e_end)) {
         // ---- this chunk's edges: lane gl of the group owns edge e + gl
@@ -136,7 +138,7 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
                 float ww = 1.f;
                 if (OP != GNNPRE_OP_SAGE_MEAN) ww = __shfl_sync(kFull, w, t & (G - 1), G);
 #pragma unroll
-                for (int v = 0; v < V; ++v) fma4(acc[v], ww, x[u][v]);
+                for (int v = 0; v < V; ++v) kahan_fma4(tot[v], cmp[v], ww, x[u][v]);
                 if (ok) open = true;
                 if (ok && (craw[u] & kRowEndBit)) {
                     // last edge of a row: all lanes of the group arrive here together
@@ -155,22 +157,16 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         const int q = gl + v * G;
-                        kahan4(tot[v], cmp[v], acc[v]);
                         if (q < a.f4) {
                             float4 o = tot[v];
                             o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
                             *reinterpret_cast<float4*>(dst + 4 * q) = o;
                         }
-                        acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                     open = false;
                 }
             }
-        }
-#pragma unroll
-        for (int v = 0; v < V; ++v) {  // fold the chunk into the row's running sum
-            kahan4(tot[v], cmp[v], acc[v]);
-            acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
         }
         rank += __popc(ends);
         e += G;
