@@ -205,13 +205,14 @@ def gnnpre_propagate(plan: Plan, X: torch.Tensor, K: int, out: Sequence[torch.Te
         else:
             out = [torch.empty((n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
     assert len(out) == K
-    ldo = out[0].stride(0)
+    ldo = out[0].stride(0) if K > 0 else F
     for o in out:
         assert o.dtype == torch.float32 and o.shape == (n, F) and o.stride(1) == 1 and o.stride(0) == ldo
         assert o.is_cuda == out[0].is_cuda
-    ptrs = (ctypes.c_void_p * K)(*[o.data_ptr() for o in out])
+    ptrs = (ctypes.c_void_p * max(K, 1))(*[o.data_ptr() for o in out])
     stats = gnnpre_stats_t() if want_stats else None
-    _check(_lib.gnnpre_propagate(plan.handle, X.data_ptr(), X.stride(0), _mem_of(X), K, ptrs, ldo, _mem_of(out[0]),
+    _check(_lib.gnnpre_propagate(plan.handle, X.data_ptr(), X.stride(0), _mem_of(X), K, ptrs, ldo,
+                                 _mem_of(out[0]) if K > 0 else _mem_of(X),
                                  _stream_ptr(stream), ctypes.byref(stats) if want_stats else None),
            "gnnpre_propagate")
     return list(out), stats

@@ -145,6 +145,7 @@ struct gnnpre_plan {
     gnnpre::DevBuf<uint32_t> colx;            // column | row-end bit, |E| entries (device-resident structure)
     gnnpre::PinnedBuf<uint32_t> colx_host;    // same, when the structure lives on the host
     gnnpre::DevBuf<uint32_t> colx_stage[2];   // double-buffered edge blocks (host structure)
+    int64_t stage_holds[2] = {-1, -1};        // which block each staging buffer currently holds
     // decomposition
     std::vector<gnnpre::Block> blocks;
     gnnpre::DevBuf<gnnpre::Segment> segments;  // num_segments + 1 (the sentinel carries the end edge)

@@ -259,3 +259,54 @@ def test_graph_without_edges(B):
         torch.cuda.synchronize()
         torch.testing.assert_close(outs[0], want, rtol=1e-6, atol=0)
         plan.close()
+
+
+# ------------------------------------------------------------------ streamed operands
+
+@pytest.mark.parametrize("csr_on_host,x_on_host,out_on_host", [(False, True, True), (True, True, True),
+                                                               (False, False, True), (True, True, False)])
+@pytest.mark.parametrize("op", OPS)
+def test_streamed_equals_resident_bitwise(B, op, csr_on_host, x_on_host, out_on_host):
+    """Host-resident operands travel through the same kernels in the same order, so for the same
+    (b, c) and segment size the result is bit-identical to the device-resident run."""
+    g = gi.rmat(30000, 250000, 13, directed_candidates=True)
+    F, K = 48, 3
+    drp, dci = dev(g)
+    X = gi.normal_matrix(g.n, F, 5, device="cuda")
+    for b, c in ((1, 1), (5, 1), (3, 3), (2, 12)):
+        ref_plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c,
+                                       segment_edges=64)
+        ref, _ = B.gnnpre_propagate(ref_plan, X, K)
+        torch.cuda.synchronize()
+        rp, ci = (g.rowptr.pin_memory(), g.colidx.pin_memory()) if csr_on_host else (drp, dci)
+        plan = B.gnnpre_build_plan(rp, ci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c, segment_edges=64,
+                                   operands_mem=B.GNNPRE_MEM_HOST)
+        assert plan.info()["structure_mem"] == (1 if csr_on_host else 0)
+        Xin = X.cpu().pin_memory() if x_on_host else X
+        ldo = F + 4
+        if out_on_host:
+            obuf = [torch.full((g.n, ldo), -3.0).pin_memory() for _ in range(K)]
+        else:
+            obuf = [torch.full((g.n, ldo), -3.0, device="cuda") for _ in range(K)]
+        for rep in range(2):  # the second call reuses the plan's staging buffers
+            outs, st = B.gnnpre_propagate(plan, Xin, K, [o[:, :F] for o in obuf], want_stats=True)
+            torch.cuda.synchronize()
+            for k in range(K):
+                assert torch.equal(outs[k].cpu(), ref[k].cpu()), (b, c, k, rep)
+                assert bool((obuf[k][:, F:] == -3.0).all())
+            assert st.d2h_bytes == (4 * g.n * F * K if out_on_host else 0)
+            assert st.h2d_bytes >= (4 * g.n * F if x_on_host else 0)
+        plan.close()
+        ref_plan.close()
+
+
+def test_streamed_pageable_host_memory_and_check_against_oracle(B):
+    g = gi.erdos_renyi(2000, 9000, 14)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    X = gi.normal_matrix(g.n, 32, 6)  # ordinary pageable host tensors
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, 0, 32, force_blocks=3, force_col_slabs=2,
+                               operands_mem=B.GNNPRE_MEM_HOST)
+    outs = [torch.empty(g.n, 32) for _ in range(2)]
+    B.gnnpre_propagate(plan, X, 2, outs)
+    check_all_hops(0, 0.0, rp, ci, X.numpy(), outs)
+    plan.close()
