@@ -137,9 +137,12 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
                 const bool ok = t < cnt;
                 float ww = 1.f;
                 if (OP != GNNPRE_OP_SAGE_MEAN) ww = __shfl_sync(kFull, w, t & (G - 1), G);
+                if (ok) {  // a padding step must not touch the compensated sum: results stay independent
+                           // of which other segment shares the warp
 #pragma unroll
-                for (int v = 0; v < V; ++v) kahan_fma4(tot[v], cmp[v], ww, x[u][v]);
-                if (ok) open = true;
+                    for (int v = 0; v < V; ++v) kahan_fma4(tot[v], cmp[v], ww, x[u][v]);
+                    open = true;
+                }
                 if (ok && (craw[u] & kRowEndBit)) {
                     // last edge of a row: all lanes of the group arrive here together
                     const int row = __shfl_sync(gmask, my_row, gshift + t);

@@ -278,6 +278,13 @@ def test_streamed_equals_resident_bitwise(B, op, csr_on_host, x_on_host, out_on_
                                        segment_edges=64)
         ref, _ = B.gnnpre_propagate(ref_plan, X, K)
         torch.cuda.synchronize()
+        pb_plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c,
+                                      segment_edges=64, flags=B.GNNPRE_FLAG_LAUNCH_PER_BLOCK)
+        pb, _ = B.gnnpre_propagate(pb_plan, X, K)  # one launch per block: same bits as one launch per hop
+        torch.cuda.synchronize()
+        for k in range(K):
+            assert torch.equal(pb[k], ref[k])
+        pb_plan.close()
         rp, ci = (g.rowptr.pin_memory(), g.colidx.pin_memory()) if csr_on_host else (drp, dci)
         plan = B.gnnpre_build_plan(rp, ci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c, segment_edges=64,
                                    operands_mem=B.GNNPRE_MEM_HOST)
