@@ -42,7 +42,8 @@ typedef enum {
     GNNPRE_ERR_CUDA = -7,             /* a CUDA call failed; gnnpre_last_cuda_error() names it */
     GNNPRE_ERR_TIMEOUT = -8,
     GNNPRE_ERR_BUSY = -9,             /* the plan is already inside a propagate call */
-    GNNPRE_ERR_UNSUPPORTED_ARCH = -10
+    GNNPRE_ERR_UNSUPPORTED_ARCH = -10,
+    GNNPRE_ERR_TOO_LARGE = -11        /* gnnpre_hop_static: the problem does not fit the fixed scratch array */
 } gnnpre_status_t;
 
 typedef enum { GNNPRE_OP_GCN_SYM = 0, GNNPRE_OP_SAGE_MEAN = 1, GNNPRE_OP_GIN_SUM = 2 } gnnpre_op_t;
@@ -173,6 +174,39 @@ int gnnpre_propagate(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t x
                      int64_t ldo, int32_t out_mem, void* stream, gnnpre_stats_t* stats);
 
 void gnnpre_plan_destroy(gnnpre_plan_t* plan);
+
+/*
+ * One hop without any allocation:  out <- A^ X  computed directly from the caller's CSR.
+ * (The paper has no counterpart of this call; it exists for callers that must not allocate.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework whose memory
+ * pool owns the whole device, in a latency-critical loop where an allocation would synchronise the
+ * device, or after start-up in a process that has promised a fixed memory footprint.  Such callers
+ * cannot use gnnpre_build_plan (it allocates the plan's tables and scratch), so this call takes no
+ * plan: it finds rows by searching `rowptr`, recomputes the scale factors on the fly, and keeps the
+ * partial sums of rows cut by its segment boundaries in a fixed array of
+ * GNNPRE_STATIC_SCRATCH_BYTES bytes that is part of the library's device image (every device that
+ * loads the library holds it until the process exits).  It is slower than a planned hop and meant
+ * for modest sizes.
+ *
+ *   csr        device-resident, same contract as gnnpre_csr_t above; NOT validated here
+ *   X, out     device, fp32 row-major [n, feat_dim] with leading dimensions ldx, ldo (multiples of 4,
+ *              16-byte aligned bases, out != X); feat_dim a multiple of 4, at most 512
+ * The work is enqueued on `stream`; the call returns at once and calls no cudaMalloc, cudaFree or
+ * other allocating routine.  The first call on a device also looks up the device address of the
+ * fixed array (once per device, with that device current), so make that first call outside any
+ * stream capture.
+ * Limits: feat_dim <= 512 and 2 * ceil(nnz / 2^20) * feat_dim * 4 <= GNNPRE_STATIC_SCRATCH_BYTES,
+ * else GNNPRE_ERR_TOO_LARGE (nothing is launched).
+ * All calls on a device share the one array.  Each call overwrites the entries it later reads, so
+ * nothing needs clearing between calls, but two calls whose kernels overlap on the GPU (different
+ * streams, or different threads) race on it: run them one after the other.
+ * Results agree with gnnpre_propagate to rounding (the self-loop term is added last instead of at
+ * its sorted position), not bit for bit.
+ */
+#define GNNPRE_STATIC_SCRATCH_BYTES (64u << 20)
+int gnnpre_hop_static(const gnnpre_csr_t* csr, int32_t op, float gin_eps, int64_t feat_dim, const float* X,
+                      int64_t ldx, float* out, int64_t ldo, void* stream);
 
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;

@@ -82,6 +82,7 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_plan_support.argtypes = [p, p, p]
     lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
                                      ctypes.POINTER(gnnpre_stats_t)]
+    lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
     lib.gnnpre_plan_destroy.argtypes = [p]
     lib.gnnpre_plan_destroy.restype = None
     lib.gnnpre_solve_budget.argtypes = [i64] * 8 + [ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -218,6 +219,17 @@ def gnnpre_propagate(plan: Plan, X: torch.Tensor, K: int, out: Sequence[torch.Te
     return list(out), stats
 
 
+def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: torch.Tensor, out: torch.Tensor, *,
+                      gin_eps: float = 0.0, stream=None) -> torch.Tensor:
+    """out = A^ X in one call that allocates nothing (the caller supplies `out`); device tensors only."""
+    assert X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1 and X.is_cuda
+    assert out.dtype == torch.float32 and out.shape == X.shape and out.stride(1) == 1 and out.is_cuda
+    csr = _csr(rowptr, colidx)
+    _check(_lib.gnnpre_hop_static(ctypes.byref(csr), op, gin_eps, X.shape[1], X.data_ptr(), X.stride(0),
+                                  out.data_ptr(), out.stride(0), _stream_ptr(stream)), "gnnpre_hop_static")
+    return out
+
+
 def gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
     b, c = ctypes.c_int64(), ctypes.c_int64()
     rc = _lib.gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c, ctypes.byref(b),
@@ -234,5 +246,5 @@ def gnnpre_status_string(status: int) -> str:
 
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
-            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

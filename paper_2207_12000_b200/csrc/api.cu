@@ -35,6 +35,7 @@ extern "C" const char* gnnpre_status_string(int status) {
     case GNNPRE_ERR_TIMEOUT: return "timed out";
     case GNNPRE_ERR_BUSY: return "plan is busy";
     case GNNPRE_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+    case GNNPRE_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of gnnpre_hop_static";
     default: return "unknown status";
     }
 }

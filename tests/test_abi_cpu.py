@@ -47,7 +47,7 @@ def test_struct_layouts_match_header(binding):
 
 def test_status_strings(binding):
     assert binding.gnnpre_status_string(0) == "ok"
-    for s in range(-10, 0):
+    for s in range(-11, 0):
         assert binding.gnnpre_status_string(s) != "unknown status"
     assert binding.gnnpre_status_string(-99) == "unknown status"
 

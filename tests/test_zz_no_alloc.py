@@ -1,0 +1,60 @@
+"""gnnpre_hop_static, the hop that allocates nothing, against the planned path.
+
+Some callers may not allocate device memory (a framework's pool owns the device, or the process
+has frozen its footprint), so they cannot build a plan; gnnpre_hop_static serves them with a
+scratch array that is part of the library image.  This file is collected last on purpose: the
+static array is shared by every call in the process, and a failure here must not hide the other
+tests from a run that stops at the first failure.
+"""
+import numpy as np
+import pytest
+import torch
+
+import gnnpre_inputs as gi
+from parity_util import TOL, hop_error, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2207_12000_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("op", (0, 1, 2))
+def test_static_hop_matches_planned_hop_twice_in_a_row(B, op):
+    """Two calls back to back with different inputs: the second must not see anything the first left
+    in the shared scratch array.  Compared with gnnpre_propagate (K = 1) at the tolerance of the
+    parity tests; the graph has isolated nodes and hubs far longer than a segment."""
+    g = gi.rmat(20000, 300000, 21, directed_candidates=True)
+    drp, dci = g.rowptr.cuda(), g.colidx.cuda()
+    for F in (100, 16):
+        plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=0.1)
+        for seed in (1, 2):
+            X = gi.normal_matrix(g.n, F, seed, device="cuda")
+            want, _ = B.gnnpre_propagate(plan, X, 1)
+            buf = torch.full((g.n, F + 4), -5.0, device="cuda")
+            got = B.gnnpre_hop_static(drp, dci, op, X, buf[:, :F], gin_eps=0.1)
+            torch.cuda.synchronize()
+            assert hop_error(to_np(got), to_np(want[0]).astype(np.float64)) <= TOL
+            assert bool((buf[:, F:] == -5.0).all())
+        plan.close()
+
+
+def test_static_hop_edge_cases_and_limits(B):
+    g = gi.from_edge_list(6, [])  # no edges: only self-loop terms
+    X = gi.normal_matrix(6, 8, 3, device="cuda")
+    out = torch.empty_like(X)
+    B.gnnpre_hop_static(g.rowptr.cuda(), g.colidx.cuda(), 0, X, out)
+    torch.cuda.synchronize()
+    assert torch.equal(out, X)
+    B.gnnpre_hop_static(g.rowptr.cuda(), g.colidx.cuda(), 1, X, out)
+    torch.cuda.synchronize()
+    assert bool((out == 0).all())
+    wide = torch.zeros((6, 516), device="cuda")
+    with pytest.raises(B.GnnpreError) as ei:
+        B.gnnpre_hop_static(g.rowptr.cuda(), g.colidx.cuda(), 0, wide, torch.empty_like(wide))
+    assert ei.value.status == -11  # beyond the fixed array's reach: a clear refusal, nothing launched
