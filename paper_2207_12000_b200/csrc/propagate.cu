@@ -55,7 +55,12 @@ __device__ __forceinline__ void kahan_fma4(float4& sum, float4& comp, float w, c
     kahan_fma1(sum.w, comp.w, w, x.w);
 }
 
-__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) { kahan_fma1(sum, comp, 1.f, x); }
+__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) {
+    const float y = x - comp;
+    const float t = sum + y;
+    comp = (t - sum) - y;
+    sum = t;
+}
 
 __device__ __forceinline__ void kahan4(float4& sum, float4& comp, const float4& x) {
     kahan1(sum.x, comp.x, x.x);
@@ -67,8 +72,18 @@ __device__ __forceinline__ void kahan4(float4& sum, float4& comp, const float4& 
 constexpr int kThreads = 256;
 
 // G lanes per segment, V float4 per lane (row width <= 4*G*V floats), U rows in flight per lane.
+//
+// Accumulation: the U rows of one step are added in a short plain fp32 chain, and that partial sum
+// enters the row's running sum by a compensated (Kahan) addition, so the rounding error of a row
+// stays at a few ulps of sum_j |w_j x_j| whatever its degree, at ~2 extra instructions per edge.
+#ifndef GNNPRE_SEG_U
+#define GNNPRE_SEG_U 8
+#endif
+#ifndef GNNPRE_SEG_MIN_BLOCKS
+#define GNNPRE_SEG_MIN_BLOCKS 3
+#endif
 template <int G, int V, int U, int OP, bool HAS_EMPTY>
-__global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
+__global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (G - 1);
@@ -87,32 +102,43 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
         slot_head = g.slot_head;
         slot_tail = g.slot_tail;
     }
-    bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
-    bool open = false;                   // edges accumulated since the last store
-    float4 tot[V], cmp[V];               // the row's running sum and its compensation
+    // Lane gl owns float4 columns gl, gl + G, ...; lanes beyond the row's width re-read column 0 so
+    // that every load is unconditional and in bounds (their sums are never stored).
+    bool on[V];
+    const float4* xlane[V];
+    const uint32_t ldx4 = (uint32_t)(a.ldx >> 2);
 #pragma unroll
-    for (int v = 0; v < V; ++v) tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int v = 0; v < V; ++v) {
+        const int q = gl + v * G;
+        on[v] = q < a.f4;
+        xlane[v] = reinterpret_cast<const float4*>(a.x) + (on[v] ? q : 0);
+    }
+    bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
+    bool open = false;                   // the last edge seen so far did not end its row
+    float4 acc[V], tot[V], cmp[V];       // this step's plain sum; the row's running sum and its compensation
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
 
     while (__any_sync(kFull, e < e_end)) {
-        // ---- this chunk's edges: lane gl of the group owns edge e + gl
+        // ---- this chunk's edges: lane gl of the group owns edge e + gl; lanes past the end hold 0,
+        // a valid column without a row-end mark
         const int64_t left = e_end - e;
         const int cnt = left >= G ? G : (left > 0 ? (int)left : 0);
         uint32_t c = 0;
         if (gl < cnt) c = a.colx[e + gl - a.colx_base];
         const unsigned ends = (__ballot_sync(kFull, (c & kRowEndBit) != 0) >> gshift) & glow;
-        const int my_rank = rank + __popc(ends & ((1u << gl) - 1u));
-        const int col = (int)(c & ~kRowEndBit);
-        int my_row = my_rank;
+        int my_row = rank + __popc(ends & ((1u << gl) - 1u));
         float my_r = 1.f, w = 1.f;
         if (c & kRowEndBit) {
-            if (HAS_EMPTY) my_row = a.nzrows[my_rank];
+            if (HAS_EMPTY) my_row = a.nzrows[my_row];
             if (OP != GNNPRE_OP_GIN_SUM) my_r = a.rscale[my_row];
         }
         if (OP == GNNPRE_OP_GCN_SYM) {
-            if (gl < cnt) w = a.cscale[col];
+            w = a.cscale[c & ~kRowEndBit];
         } else if (OP == GNNPRE_OP_GIN_SUM) {
-            w = col == my_row ? a.diag_weight : 1.f;  // every row owns its self-loop, so rank == row
+            w = (int)(c & ~kRowEndBit) == my_row ? a.diag_weight : 1.f;  // every row owns its self-loop: rank == row
         }
+        if (cnt > 0) open = (__shfl_sync(gmask, c, gshift + cnt - 1) & kRowEndBit) == 0;
         const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
 
         // ---- gather and accumulate, U rows in flight
@@ -121,30 +147,32 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
             uint32_t craw[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
-                const int t = t0 + u;  // may run past G - 1 in the last step: the shuffle wraps, `ok` masks it
-                craw[u] = __shfl_sync(kFull, c, t & (G - 1), G);
-                const bool ok = t < cnt;
-                const float* row = a.x + (int64_t)(craw[u] & ~kRowEndBit) * a.ldx;
+                craw[u] = __shfl_sync(kFull, c, t0 + u, G);
+                const uint64_t off = (uint64_t)(craw[u] & ~kRowEndBit) * ldx4;
 #pragma unroll
-                for (int v = 0; v < V; ++v) {
-                    const int q = gl + v * G;
-                    x[u][v] = (ok && q < a.f4) ? ld_row(row + 4 * q) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
+                for (int v = 0; v < V; ++v) x[u][v] = __ldg(xlane[v] + off);
             }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int t = t0 + u;
-                const bool ok = t < cnt;
-                float ww = 1.f;
-                if (OP != GNNPRE_OP_SAGE_MEAN) ww = __shfl_sync(kFull, w, t & (G - 1), G);
-                if (ok) {  // a padding step must not touch the compensated sum: results stay independent
-                           // of which other segment shares the warp
+                if (t < cnt) {
+                    if (OP == GNNPRE_OP_SAGE_MEAN) {
 #pragma unroll
-                    for (int v = 0; v < V; ++v) kahan_fma4(tot[v], cmp[v], ww, x[u][v]);
-                    open = true;
+                        for (int v = 0; v < V; ++v) {
+                            acc[v].x += x[u][v].x; acc[v].y += x[u][v].y;
+                            acc[v].z += x[u][v].z; acc[v].w += x[u][v].w;
+                        }
+                    } else {
+                        const float ww = __shfl_sync(gmask, w, gshift + t);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            acc[v].x = fmaf(ww, x[u][v].x, acc[v].x); acc[v].y = fmaf(ww, x[u][v].y, acc[v].y);
+                            acc[v].z = fmaf(ww, x[u][v].z, acc[v].z); acc[v].w = fmaf(ww, x[u][v].w, acc[v].w);
+                        }
+                    }
                 }
-                if (ok && (craw[u] & kRowEndBit)) {
-                    // last edge of a row: all lanes of the group arrive here together
+                if (craw[u] & kRowEndBit) {
+                    // last edge of a row (never set on a padding lane): the whole group arrives here together
                     const int row = __shfl_sync(gmask, my_row, gshift + t);
                     const float r = __shfl_sync(gmask, my_r, gshift + t);
                     float* dst;
@@ -159,15 +187,22 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
                     }
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
-                        const int q = gl + v * G;
-                        if (q < a.f4) {
+                        kahan4(tot[v], cmp[v], acc[v]);
+                        if (on[v]) {
                             float4 o = tot[v];
                             o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
-                            *reinterpret_cast<float4*>(dst + 4 * q) = o;
+                            reinterpret_cast<float4*>(dst)[gl + v * G] = o;
                         }
-                        tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
-                    open = false;
+                }
+            }
+            if (t0 < cnt) {  // this step's plain sum joins the row's compensated sum (never on a padding
+                             // step: the result must not depend on which segment shares the warp)
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    kahan4(tot[v], cmp[v], acc[v]);
+                    acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                 }
             }
         }
@@ -181,10 +216,8 @@ __global__ void __launch_bounds__(kThreads) k_segments(const SegArgs a) {
         if (slot >= 0) {
             float* dst = a.scratch + (int64_t)slot * a.scratch_ld;
 #pragma unroll
-            for (int v = 0; v < V; ++v) {
-                const int q = gl + v * G;
-                if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = tot[v];
-            }
+            for (int v = 0; v < V; ++v)
+                if (on[v]) reinterpret_cast<float4*>(dst)[gl + v * G] = tot[v];
         }
     }
 }
@@ -325,7 +358,7 @@ int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int6
         if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
         else if (a.f4 <= 8) GNNPRE_TRY((launch_segments_shape<8, 1, 8>(P, a, st)));
         else if (a.f4 <= 16) GNNPRE_TRY((launch_segments_shape<16, 1, 8>(P, a, st)));
-        else if (a.f4 <= 32) GNNPRE_TRY((launch_segments_shape<32, 1, 8>(P, a, st)));
+        else if (a.f4 <= 32) GNNPRE_TRY((launch_segments_shape<32, 1, GNNPRE_SEG_U>(P, a, st)));
         else if (a.f4 <= 64) GNNPRE_TRY((launch_segments_shape<32, 2, 4>(P, a, st)));
         else GNNPRE_TRY((launch_segments_shape<32, 4, 2>(P, a, st)));
     }
