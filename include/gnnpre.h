@@ -68,6 +68,8 @@ typedef struct {
 /* gnnpre_plan_opts_t.flags */
 #define GNNPRE_FLAG_LAUNCH_PER_BLOCK 1u /* device-resident runs: one kernel launch per edge block instead of one per hop */
 #define GNNPRE_FLAG_SKIP_VALIDATION 2u  /* trust the CSR contract (saves one pass over the graph) */
+#define GNNPRE_FLAG_NO_BULK_COPY 4u     /* gather into registers for every width (default: rows of 68..128 columns
+                                           are staged through shared memory by the bulk-copy engine); same bits */
 
 typedef struct {
     int32_t op;              /* gnnpre_op_t */

@@ -16,7 +16,7 @@ from . import build as _build
 
 GNNPRE_OP_GCN_SYM, GNNPRE_OP_SAGE_MEAN, GNNPRE_OP_GIN_SUM = 0, 1, 2
 GNNPRE_MEM_DEVICE, GNNPRE_MEM_HOST = 0, 1
-GNNPRE_FLAG_LAUNCH_PER_BLOCK, GNNPRE_FLAG_SKIP_VALIDATION = 1, 2
+GNNPRE_FLAG_LAUNCH_PER_BLOCK, GNNPRE_FLAG_SKIP_VALIDATION, GNNPRE_FLAG_NO_BULK_COPY = 1, 2, 4
 GNNPRE_MAX_HOPS = 64
 
 

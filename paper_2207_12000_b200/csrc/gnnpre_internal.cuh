@@ -152,6 +152,8 @@ struct gnnpre_plan {
     gnnpre::DevBuf<gnnpre::RowFixup> fixups;
     int64_t num_segments = 0, num_fixups = 0, num_slots = 0;
     gnnpre::DevBuf<float> scratch;  // num_slots rows of slab_width floats
+    gnnpre::DevBuf<int> dev_error;  // set by a kernel whose bounded wait ran out
+    int num_sms = 0;
     // streaming state
     gnnpre::DevBuf<float> slab[4];
     cudaStream_t s_h2d = nullptr, s_d2h = nullptr, s_compute = nullptr;
@@ -190,5 +192,7 @@ int propagate_streamed(gnnpre_plan* plan, const float* X, int64_t ldx, int32_t x
 int solve_budget(int64_t B_S, int64_t B_X, int64_t B_fixed, int64_t beta_S, int64_t beta_X, int64_t B_GPU,
                  int64_t max_b, int64_t max_c, int64_t* b_out, int64_t* c_out);
 int check_device();
+int check_device_error(gnnpre_plan* plan);  // synchronous read of plan->dev_error: GNNPRE_ERR_TIMEOUT if set
+bool uses_bulk_copy(const gnnpre_plan* plan, int32_t width);
 
 }  // namespace gnnpre

@@ -337,7 +337,15 @@ __global__ void k_gather_i32(int count, const int64_t* __restrict__ idx, const i
     if (i < count) dst[i] = src[idx[i]];
 }
 
-int32_t auto_segment_edges(int64_t slab_width) {
+int32_t auto_segment_edges(int64_t slab_width, int64_t m, bool bulk_copy, int num_sms) {
+    if (bulk_copy) {
+        // persistent warps walk whole segments with a two-stage pipeline that drains at every segment
+        // end: long segments, but at least ~4 per resident warp so the tail stays short
+        const int64_t per_warp = m / ((int64_t)std::max(num_sms, 1) * 8 * 4);
+        int32_t p = 256;
+        while ((int64_t)p * 2 <= per_warp && p < 4096) p *= 2;
+        return p;
+    }
     // about 32 Ki gathered floats per segment, a power of two between 32 and 4096 edges
     int64_t L = 32768 / std::max<int64_t>(slab_width, 4);
     int32_t p = 32;
@@ -377,6 +385,15 @@ int solve_budget(int64_t B_S, int64_t B_X, int64_t B_fixed, int64_t beta_S, int6
     return GNNPRE_OK;
 }
 
+int check_device_error(gnnpre_plan* P) {
+    if (!P->dev_error.p) return GNNPRE_OK;
+    int h = 0;
+    GNNPRE_CUDA(cudaMemcpy(&h, P->dev_error.p, sizeof(int), cudaMemcpyDeviceToHost));
+    if (h == 0) return GNNPRE_OK;
+    GNNPRE_CUDA(cudaMemset(P->dev_error.p, 0, sizeof(int)));
+    return GNNPRE_ERR_TIMEOUT;
+}
+
 int check_device() {
     int dev = 0;
     GNNPRE_CUDA(cudaGetDevice(&dev));
@@ -398,7 +415,7 @@ gnnpre_plan::~gnnpre_plan() {
 int64_t gnnpre_plan::device_bytes() const {
     size_t t = deg.bytes() + rscale.bytes() + cscale.bytes() + nzrows.bytes() + emptyrows.bytes() + rowptr_t.bytes() +
                colx.bytes() + colx_stage[0].bytes() + colx_stage[1].bytes() + segments.bytes() + fixups.bytes() +
-               scratch.bytes();
+               scratch.bytes() + dev_error.bytes();
     for (const auto& s : slab) t += s.bytes();
     return (int64_t)t;
 }
@@ -561,7 +578,10 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     P->c = (int32_t)c;
     P->slab_width = 4 * ((F + 4 * c - 1) / (4 * c));
     if (P->slab_width * (c - 1) >= F) return GNNPRE_ERR_INVALID_ARG;  // a slab would be empty
-    P->segment_edges = opts->segment_edges > 0 ? opts->segment_edges : auto_segment_edges(P->slab_width);
+    GNNPRE_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
+    P->segment_edges = opts->segment_edges > 0
+                           ? opts->segment_edges
+                           : auto_segment_edges(P->slab_width, m, uses_bulk_copy(P, (int32_t)P->slab_width), P->num_sms);
     if (P->segment_edges < 1) return GNNPRE_ERR_INVALID_ARG;
 
     // ---- block table: block l = edges [floor(l m / b), floor((l+1) m / b))
@@ -651,6 +671,8 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     }
 
     GNNPRE_TRY(P->scratch.alloc((size_t)P->num_slots * (size_t)P->slab_width));
+    GNNPRE_TRY(P->dev_error.alloc(1));
+    GNNPRE_CUDA(cudaMemset(P->dev_error.p, 0, sizeof(int)));
 
     // ---- a host-resident structure keeps E in pinned memory and streams it block by block
     if (P->structure_mem == GNNPRE_MEM_HOST) {

@@ -36,25 +36,8 @@ struct SegArgs {
     float diag_weight;  // GIN: 1 + eps
 };
 
-__device__ __forceinline__ float4 ld_row(const float* p) { return __ldg(reinterpret_cast<const float4*>(p)); }
-
-// Compensated (Kahan) summation in fp32: the pair (sum, comp) absorbs w*x with the low-order bits
-// that the addition drops carried in comp, so the error of a row's sum stays at a few ulps of
-// sum_j |w_j x_j| whatever the degree.  The kernel is bound by memory, not by these extra adds.
-__device__ __forceinline__ void kahan_fma1(float& sum, float& comp, float w, float x) {
-    const float y = fmaf(w, x, -comp);
-    const float t = sum + y;
-    comp = (t - sum) - y;
-    sum = t;
-}
-
-__device__ __forceinline__ void kahan_fma4(float4& sum, float4& comp, float w, const float4& x) {
-    kahan_fma1(sum.x, comp.x, w, x.x);
-    kahan_fma1(sum.y, comp.y, w, x.y);
-    kahan_fma1(sum.z, comp.z, w, x.z);
-    kahan_fma1(sum.w, comp.w, w, x.w);
-}
-
+// Compensated (Kahan) addition of x into the pair (sum, comp): the low-order bits that the addition
+// drops are carried in comp.
 __device__ __forceinline__ void kahan1(float& sum, float& comp, float x) {
     const float y = x - comp;
     const float t = sum + y;
@@ -222,6 +205,8 @@ __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(co
     }
 }
 
+#include "segments_tma.cuh"
+
 struct FixArgs {
     const RowFixup* fix;
     int64_t fix_lo, fix_hi;
@@ -321,6 +306,38 @@ int launch_segments_shape(const gnnpre_plan* P, const SegArgs& a, cudaStream_t s
     return GNNPRE_OK;
 }
 
+// Bulk-copy variant: one persistent CTA per SM, as many warps as two stages of 32 rows each fit
+// into the SM's shared memory (at most 8).
+constexpr size_t kTmaSmemBudget = 227 * 1024 - 1024;
+
+int tma_warps(int32_t f4) {
+    const size_t per_warp = (size_t)kTmaStages * kTmaRows * 16u * (size_t)f4;
+    return (int)std::min<size_t>(kTmaMaxWarps, kTmaSmemBudget / per_warp);
+}
+
+template <int OP, bool HAS_EMPTY>
+int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
+    const int nwarps = tma_warps(a.f4);
+    const size_t smem = (size_t)nwarps * kTmaStages * kTmaRows * 16u * (size_t)a.f4;
+    auto kernel = k_segments_tma<OP, HAS_EMPTY>;
+    GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const int64_t nseg = a.seg_hi - a.seg_lo;
+    const unsigned grid = (unsigned)std::min<int64_t>(P->num_sms, (nseg + nwarps - 1) / nwarps);
+    kernel<<<grid, nwarps * 32, smem, st>>>(a, P->dev_error.p);
+    GNNPRE_CUDA(cudaGetLastError());
+    return GNNPRE_OK;
+}
+
+int launch_segments_tma(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
+    switch (P->op) {
+    case GNNPRE_OP_GCN_SYM: return launch_segments_tma_op<GNNPRE_OP_GCN_SYM, false>(P, a, st);
+    case GNNPRE_OP_GIN_SUM: return launch_segments_tma_op<GNNPRE_OP_GIN_SUM, false>(P, a, st);
+    default:
+        return P->rows_all_nonempty ? launch_segments_tma_op<GNNPRE_OP_SAGE_MEAN, false>(P, a, st)
+                                    : launch_segments_tma_op<GNNPRE_OP_SAGE_MEAN, true>(P, a, st);
+    }
+}
+
 template <int G, int V>
 int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
     const int64_t groups = a.fix_hi - a.fix_lo;
@@ -333,6 +350,12 @@ int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
 constexpr int kMaxTile = 512;  // columns one launch covers (G = 32, V = 4)
 
 }  // namespace
+
+// Rows of 68..128 columns (17..32 float4) go through the bulk-copy kernel unless the plan says otherwise.
+bool uses_bulk_copy(const gnnpre_plan* P, int32_t width) {
+    const int32_t f4 = width / 4;
+    return !(P->flags & GNNPRE_FLAG_NO_BULK_COPY) && f4 > 16 && f4 <= 32 && tma_warps(f4) >= 2;
+}
 
 int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int64_t seg_hi, cudaStream_t st) {
     if (seg_hi <= seg_lo) return GNNPRE_OK;
@@ -355,7 +378,8 @@ int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int6
         a.nzrows = P->nzrows.p;
         a.f4 = w / 4;
         a.diag_weight = 1.0f + P->gin_eps;
-        if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
+        if (uses_bulk_copy(P, w)) GNNPRE_TRY(launch_segments_tma(P, a, st));
+        else if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
         else if (a.f4 <= 8) GNNPRE_TRY((launch_segments_shape<8, 1, 8>(P, a, st)));
         else if (a.f4 <= 16) GNNPRE_TRY((launch_segments_shape<16, 1, 8>(P, a, st)));
         else if (a.f4 <= 32) GNNPRE_TRY((launch_segments_shape<32, 1, GNNPRE_SEG_U>(P, a, st)));
@@ -454,6 +478,7 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
     }
     if (stats) {
         if (rc == GNNPRE_OK && cudaStreamSynchronize(st) != cudaSuccess) rc = GNNPRE_ERR_CUDA;
+        if (rc == GNNPRE_OK) rc = check_device_error(P);
         if (rc == GNNPRE_OK) {
             for (int32_t k = 0; k < K; ++k) cudaEventElapsedTime(&stats->hop_ms[k], hop_ev[(size_t)k], hop_ev[(size_t)k + 1]);
             cudaEventElapsedTime(&stats->total_ms, hop_ev[0], hop_ev[(size_t)K]);

@@ -1,0 +1,251 @@
+// Segment kernel with the gathered rows staged through shared memory by the bulk-copy (TMA) engine.
+// Included by propagate.cu inside its unnamed namespace (uses SegArgs, kahan4, kRowEndBit).
+//
+// Why: the register kernel k_segments keeps at most (warps per SM) x U rows in flight, bounded by
+// the register file; a gather of 400-512 B rows at random addresses needs ~100 KB in flight per SM
+// to hide HBM/L2 latency.  Here every lane of a warp asks the copy engine for one neighbour row
+// (cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier), so a warp has up
+// to kTmaStages x 32 rows in flight and they occupy shared memory (up to ~220 KB per SM) instead of
+// registers.  The warp then sums the rows out of shared memory with conflict-free 128-bit reads.
+//
+// One CTA per SM, persistent: warp w of the grid walks segments w, w + W, w + 2W, ... (W = warps in
+// the grid), so no atomics are involved and the summation order is the same as in k_segments
+// (plain sums over steps of 8 edges, folded into the row's compensated sum): both kernels produce
+// identical bits.
+//
+// Every wait on an mbarrier is bounded: after kTmaSpinLimit polls the warp records an error in
+// a.error, drains what it has in flight (bounded as well) and leaves.
+#pragma once
+
+constexpr int kTmaStages = 2;
+constexpr int kTmaRows = 32;           // rows per stage: one chunk of edges
+constexpr int kTmaStep = 8;            // edges per plain-sum step (same as k_segments' U for G = 32, V = 1)
+constexpr int kTmaMaxWarps = 8;
+constexpr uint32_t kTmaSpinLimit = 1u << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+// true once the phase with the given parity has completed
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return done != 0;
+}
+
+// Bounded wait; false if the limit ran out.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+    for (uint32_t i = 0; i < kTmaSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+
+// bytes: a multiple of 16; dst (shared) and src (global) 16-byte aligned
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+
+// Per-stage bookkeeping a warp keeps in registers between issuing a chunk and summing it.
+struct TmaChunk {
+    uint32_t c;      // this lane's column entry (row-end mark in bit 31); 0 on padding lanes
+    unsigned ends;   // row-end marks of the chunk, bit t = edge t
+    int cnt;         // edges in the chunk
+    int row;         // row of this lane's edge (valid where it ends a row; everywhere for GIN)
+    float r, w;      // row scale of that row; weight of this lane's edge
+};
+
+template <int OP, bool HAS_EMPTY>
+__global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const SegArgs a, int* error) {
+    constexpr unsigned kFull = 0xffffffffu;
+    extern __shared__ __align__(128) unsigned char tma_smem[];
+    __shared__ __align__(8) unsigned long long bars[kTmaMaxWarps][kTmaStages];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int nwarps = blockDim.x >> 5;
+    const uint32_t rb = 16u * (uint32_t)a.f4;  // bytes of one row of this column tile
+    const uint32_t stage_bytes = kTmaRows * rb;
+    unsigned char* my_smem = tma_smem + (size_t)warp * kTmaStages * stage_bytes;
+    const uint32_t smem0 = smem_u32(my_smem);
+    const uint32_t bar0 = smem_u32(&bars[warp][0]);
+    if (lane == 0) {
+#pragma unroll
+        for (int st = 0; st < kTmaStages; ++st) mbar_init(bar0 + 8u * st, 1);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+
+    uint32_t phase[kTmaStages];
+    bool inflight[kTmaStages];
+#pragma unroll
+    for (int st = 0; st < kTmaStages; ++st) {
+        phase[st] = 0;
+        inflight[st] = false;
+    }
+    bool failed = false;
+    const bool on = lane < a.f4;  // lanes beyond the row's width re-read column 0 and never store
+    const uint32_t lane_off = on ? 16u * lane : 0u;
+    const unsigned lt_mask = (1u << lane) - 1u;
+    const uint32_t ldx4 = (uint32_t)(a.ldx >> 2);
+    const float4* xbase = reinterpret_cast<const float4*>(a.x);
+
+    const int64_t W = (int64_t)gridDim.x * nwarps;
+    for (int64_t s = a.seg_lo + (int64_t)blockIdx.x * nwarps + warp; s < a.seg_hi && !failed; s += W) {
+        const Segment g = a.segs[s];
+        const int64_t e_beg = g.start, e_end = a.segs[s + 1].start;
+        const int nchunks = (int)((e_end - e_beg + kTmaRows - 1) / kTmaRows);
+        int rank_issue = g.rank;
+        const int slot_head = g.slot_head, slot_tail = g.slot_tail;
+        bool head_pending = slot_head >= 0;
+        bool open = false;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), tot = acc, cmp = acc;
+        TmaChunk ch[kTmaStages];
+
+        // ---- ask the copy engine for the rows of chunk k, into stage st
+        auto issue = [&](int k, int st) {
+            TmaChunk& m = ch[st];
+            const int64_t e0 = e_beg + (int64_t)k * kTmaRows;
+            const int64_t left = e_end - e0;
+            m.cnt = left >= kTmaRows ? kTmaRows : (int)left;
+            uint32_t c = 0;
+            if (lane < m.cnt) c = a.colx[e0 + lane - a.colx_base];
+            m.c = c;
+            m.ends = __ballot_sync(kFull, (c & kRowEndBit) != 0);
+            int row = rank_issue + __popc(m.ends & lt_mask);
+            m.r = 1.f;
+            m.w = 1.f;
+            if (c & kRowEndBit) {
+                if (HAS_EMPTY) row = a.nzrows[row];
+                if (OP != GNNPRE_OP_GIN_SUM) m.r = a.rscale[row];
+            }
+            if (OP == GNNPRE_OP_GCN_SYM) {
+                m.w = a.cscale[c & ~kRowEndBit];
+            } else if (OP == GNNPRE_OP_GIN_SUM) {
+                m.w = (int)(c & ~kRowEndBit) == row ? a.diag_weight : 1.f;
+            }
+            m.row = row;
+            rank_issue += __popc(m.ends);
+            const uint32_t bar = bar0 + 8u * st;
+            if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)m.cnt * rb);
+            __syncwarp();
+            if (lane < m.cnt)
+                bulk_copy_g2s(smem0 + st * stage_bytes + lane * rb, xbase + (uint64_t)(c & ~kRowEndBit) * ldx4, rb, bar);
+            inflight[st] = true;
+        };
+
+        // ---- a finished row (or the head part of one) leaves the warp
+        auto flush = [&](int t, const TmaChunk& m) {
+            const int row = __shfl_sync(kFull, m.row, t);
+            const float r = __shfl_sync(kFull, m.r, t);
+            float* dst;
+            float scale;
+            if (head_pending) {
+                dst = a.scratch + (int64_t)slot_head * a.scratch_ld;
+                scale = 1.f;
+                head_pending = false;
+            } else {
+                dst = a.out + (int64_t)row * a.ldo;
+                scale = r;
+            }
+            kahan4(tot, cmp, acc);
+            if (on) {
+                float4 o = tot;
+                o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
+                reinterpret_cast<float4*>(dst)[lane] = o;
+            }
+            acc = tot = cmp = make_float4(0.f, 0.f, 0.f, 0.f);
+        };
+
+        // ---- sum the rows of the chunk held by stage st
+        auto consume = [&](int st) {
+            const TmaChunk& m = ch[st];
+            if (!mbar_wait_bounded(bar0 + 8u * st, phase[st])) {
+                failed = true;
+                return;
+            }
+            phase[st] ^= 1u;
+            inflight[st] = false;
+            const unsigned char* base = my_smem + st * stage_bytes + lane_off;
+            for (int t0 = 0; t0 < m.cnt; t0 += kTmaStep) {
+                float4 x[kTmaStep];
+#pragma unroll
+                for (int u = 0; u < kTmaStep; ++u) x[u] = *reinterpret_cast<const float4*>(base + (t0 + u) * rb);
+                const unsigned step_ends = (m.ends >> t0) & ((1u << kTmaStep) - 1u);
+                if (step_ends == 0 && t0 + kTmaStep <= m.cnt) {  // no row ends here: a straight run of adds
+#pragma unroll
+                    for (int u = 0; u < kTmaStep; ++u) {
+                        if (OP == GNNPRE_OP_SAGE_MEAN) {
+                            acc.x += x[u].x; acc.y += x[u].y; acc.z += x[u].z; acc.w += x[u].w;
+                        } else {
+                            const float ww = __shfl_sync(kFull, m.w, t0 + u);
+                            acc.x = fmaf(ww, x[u].x, acc.x); acc.y = fmaf(ww, x[u].y, acc.y);
+                            acc.z = fmaf(ww, x[u].z, acc.z); acc.w = fmaf(ww, x[u].w, acc.w);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int u = 0; u < kTmaStep; ++u) {
+                        const int t = t0 + u;
+                        if (t < m.cnt) {
+                            if (OP == GNNPRE_OP_SAGE_MEAN) {
+                                acc.x += x[u].x; acc.y += x[u].y; acc.z += x[u].z; acc.w += x[u].w;
+                            } else {
+                                const float ww = __shfl_sync(kFull, m.w, t);
+                                acc.x = fmaf(ww, x[u].x, acc.x); acc.y = fmaf(ww, x[u].y, acc.y);
+                                acc.z = fmaf(ww, x[u].z, acc.z); acc.w = fmaf(ww, x[u].w, acc.w);
+                            }
+                            if ((m.ends >> t) & 1u) flush(t, m);
+                        }
+                    }
+                }
+                kahan4(tot, cmp, acc);  // this step's plain sum joins the row's compensated sum
+                acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            open = ((m.ends >> (m.cnt - 1)) & 1u) == 0;
+            __syncwarp();  // every lane is done with the stage before it is refilled
+        };
+
+        issue(0, 0);
+        if (nchunks > 1) issue(1, 1);
+        for (int k = 0; k < nchunks && !failed; k += kTmaStages) {
+            consume(0);
+            if (failed) break;
+            if (k + 2 < nchunks) issue(k + 2, 0);
+            if (k + 1 < nchunks) {
+                consume(1);
+                if (failed) break;
+                if (k + 3 < nchunks) issue(k + 3, 1);
+            }
+        }
+        if (failed) break;
+
+        if (open) {  // the row holding the last edge continues in the next segment
+            const int slot = head_pending ? slot_head : slot_tail;
+            if (slot >= 0 && on)
+                reinterpret_cast<float4*>(a.scratch + (int64_t)slot * a.scratch_ld)[lane] = tot;
+        }
+    }
+
+    if (failed) {
+        // a wait ran out: report it, let the copies still in flight land (bounded), and leave
+        if (lane == 0) atomicExch(error, 1);
+#pragma unroll
+        for (int st = 0; st < kTmaStages; ++st)
+            if (inflight[st]) (void)mbar_wait_bounded(bar0 + 8u * st, phase[st]);
+    }
+}

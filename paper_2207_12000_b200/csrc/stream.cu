@@ -175,6 +175,7 @@ int run(gnnpre_plan* P, const float* X, int64_t ldx, bool x_host, int32_t K, flo
     GNNPRE_CUDA(cudaStreamSynchronize(P->s_h2d));
     GNNPRE_CUDA(cudaStreamSynchronize(P->s_compute));
     GNNPRE_CUDA(cudaStreamSynchronize(P->s_d2h));
+    GNNPRE_TRY(check_device_error(P));
     if (stats) {
         stats->h2d_bytes = h2d;
         stats->d2h_bytes = d2h;

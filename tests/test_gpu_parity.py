@@ -317,3 +317,23 @@ def test_streamed_pageable_host_memory_and_check_against_oracle(B):
     B.gnnpre_propagate(plan, X, 2, outs)
     check_all_hops(0, 0.0, rp, ci, X.numpy(), outs)
     plan.close()
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("F", [68, 100, 128])
+def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
+    """Rows of 68..128 columns are staged through shared memory by the copy engine; the summation
+    order is the register kernel's, so the two agree bit for bit (and both agree with the oracle)."""
+    g = gi.rmat(30000, 400000, 17, directed_candidates=True)
+    drp, dci = dev(g)
+    X = gi.normal_matrix(g.n, F, 9, device="cuda")
+    for b, seg in ((1, 0), (3, 64), (2, 1000)):
+        res = []
+        for flags in (0, B.GNNPRE_FLAG_NO_BULK_COPY):
+            plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, segment_edges=seg, flags=flags)
+            outs, st = B.gnnpre_propagate(plan, X, 2, want_stats=True)
+            res.append(outs)
+            plan.close()
+        for k in range(2):
+            assert torch.equal(res[0][k], res[1][k]), (b, seg, k)
+    check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[0])
