@@ -17,10 +17,20 @@
 // a.error, drains what it has in flight (bounded as well) and leaves.
 #pragma once
 
-constexpr int kTmaStages = 2;
-constexpr int kTmaRows = 32;           // rows per stage: one chunk of edges
-constexpr int kTmaStep = 8;            // edges per plain-sum step (same as k_segments' U for G = 32, V = 1)
-constexpr int kTmaMaxWarps = 8;
+#ifndef GNNPRE_TMA_STAGES
+#define GNNPRE_TMA_STAGES 4
+#endif
+#ifndef GNNPRE_TMA_ROWS
+#define GNNPRE_TMA_ROWS 16
+#endif
+#ifndef GNNPRE_TMA_WARPS
+#define GNNPRE_TMA_WARPS 8
+#endif
+constexpr int kTmaStages = GNNPRE_TMA_STAGES;  // chunks a warp keeps in flight
+constexpr int kTmaRows = GNNPRE_TMA_ROWS;      // rows per stage = edges per chunk (8, 16 or 32)
+constexpr int kTmaStep = 8;                    // edges per plain-sum step (same as k_segments' U for G = 32, V = 1)
+constexpr int kTmaMaxWarps = GNNPRE_TMA_WARPS;
+static_assert(kTmaRows % kTmaStep == 0 && kTmaRows <= 32, "a chunk is a whole number of steps and fits one warp");
 constexpr uint32_t kTmaSpinLimit = 1u << 22;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -110,6 +120,9 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
         const int64_t e_beg = g.start, e_end = a.segs[s + 1].start;
         const int nchunks = (int)((e_end - e_beg + kTmaRows - 1) / kTmaRows);
         int rank_issue = g.rank;
+        // column entries of the chunk that will be issued next, fetched one chunk ahead
+        uint32_t c_next = 0;
+        if (lane < kTmaRows && e_beg + lane < e_end) c_next = a.colx[e_beg + lane - a.colx_base];
         const int slot_head = g.slot_head, slot_tail = g.slot_tail;
         bool head_pending = slot_head >= 0;
         bool open = false;
@@ -122,8 +135,9 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
             const int64_t e0 = e_beg + (int64_t)k * kTmaRows;
             const int64_t left = e_end - e0;
             m.cnt = left >= kTmaRows ? kTmaRows : (int)left;
-            uint32_t c = 0;
-            if (lane < m.cnt) c = a.colx[e0 + lane - a.colx_base];
+            const uint32_t c = c_next;
+            c_next = 0;
+            if (lane < kTmaRows && e0 + kTmaRows + lane < e_end) c_next = a.colx[e0 + kTmaRows + lane - a.colx_base];
             m.c = c;
             m.ends = __ballot_sync(kFull, (c & kRowEndBit) != 0);
             int row = rank_issue + __popc(m.ends & lt_mask);
@@ -220,16 +234,16 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
             __syncwarp();  // every lane is done with the stage before it is refilled
         };
 
-        issue(0, 0);
-        if (nchunks > 1) issue(1, 1);
+#pragma unroll
+        for (int st = 0; st < kTmaStages; ++st)
+            if (st < nchunks) issue(st, st);
         for (int k = 0; k < nchunks && !failed; k += kTmaStages) {
-            consume(0);
-            if (failed) break;
-            if (k + 2 < nchunks) issue(k + 2, 0);
-            if (k + 1 < nchunks) {
-                consume(1);
-                if (failed) break;
-                if (k + 3 < nchunks) issue(k + 3, 1);
+#pragma unroll
+            for (int st = 0; st < kTmaStages; ++st) {
+                if (k + st < nchunks && !failed) {
+                    consume(st);
+                    if (!failed && k + st + kTmaStages < nchunks) issue(k + st + kTmaStages, st);
+                }
             }
         }
         if (failed) break;
