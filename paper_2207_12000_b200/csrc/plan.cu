@@ -341,7 +341,7 @@ int32_t auto_segment_edges(int64_t slab_width, int64_t m, bool bulk_copy, int nu
     if (bulk_copy) {
         // persistent warps walk whole segments with a two-stage pipeline that drains at every segment
         // end: long segments, but at least ~4 per resident warp so the tail stays short
-        const int64_t per_warp = m / ((int64_t)std::max(num_sms, 1) * 8 * 4);
+        const int64_t per_warp = m / ((int64_t)std::max(num_sms, 1) * 16 * 4);
         int32_t p = 256;
         while ((int64_t)p * 2 <= per_warp && p < 4096) p *= 2;
         return p;

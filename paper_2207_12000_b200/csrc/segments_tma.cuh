@@ -18,13 +18,13 @@
 #pragma once
 
 #ifndef GNNPRE_TMA_STAGES
-#define GNNPRE_TMA_STAGES 4
+#define GNNPRE_TMA_STAGES 2
 #endif
 #ifndef GNNPRE_TMA_ROWS
 #define GNNPRE_TMA_ROWS 16
 #endif
 #ifndef GNNPRE_TMA_WARPS
-#define GNNPRE_TMA_WARPS 8
+#define GNNPRE_TMA_WARPS 16
 #endif
 constexpr int kTmaStages = GNNPRE_TMA_STAGES;  // chunks a warp keeps in flight
 constexpr int kTmaRows = GNNPRE_TMA_ROWS;      // rows per stage = edges per chunk (8, 16 or 32)
