@@ -100,6 +100,25 @@ class ClockSampler:
                 "samples": len(self.rows)}
 
 
+def profiled_traffic(workload_name):
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None when there is
+    none for this workload or the kernel sources have changed since it was taken."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", f"k_segments_tma_{workload_name}_dram.md")
+    if not os.path.exists(path):
+        return None
+    text = open(path).read()
+    t = re.search(r"traffic_bytes_per_launch:\s*(\d+)", text)
+    h = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
+    if not t or not h:
+        return None
+    cur = hashlib.sha256()
+    for f in ("propagate.cu", "segments_tma.cuh"):
+        cur.update(open(os.path.join(ROOT, "paper_2207_12000_b200", "csrc", f), "rb").read())
+    return int(t.group(1)) if cur.hexdigest() == h.group(1) else None
+
+
 def byte_model(n, m, F):
     """Algorithmic bytes of one hop.  gather: every neighbour row comes from memory once per edge;
     min: every matrix is touched once."""
@@ -251,8 +270,13 @@ def main():
     launches_per_hop = seg_launches / (args.steps * K)
     seg_launch_ms = seg_ms / max(1, seg_launches)
     achieved = gather_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9
+    traffic = profiled_traffic(w.name) if args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": None,
+                "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": traffic,
+                "dram_achieved": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9,
+                "dram_frac": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9 / peak,
+                "model": "achieved = gather model: every neighbour row fetched once per edge, 4|E|F + 4nF + 4|E| + 16n "
+                         "bytes per hop; L2 hits make it exceed the DRAM peak; dram_achieved = ncu DRAM bytes / time",
                 "kernel": "k_segments", "kernel_ms_per_launch": seg_launch_ms,
                 "algorithmic_bytes_per_launch": gather_b / launches_per_hop,
                 "achieved_min_model": least_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9,
