@@ -45,6 +45,7 @@ def parse():
     ap.add_argument("--blocks", type=int, default=-1, help="override the workload's block count")
     ap.add_argument("--per-block-launch", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
+    ap.add_argument("--budget-gb", type=float, default=0.0, help="device-memory budget B_GPU of the streamed plan (0 = free memory)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -289,9 +290,13 @@ def main():
             Xh = torch.empty((g.n, F), dtype=torch.float32, pin_memory=True)
             Xh.copy_(X)
             outs_h = [torch.empty((g.n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
-            hplan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
+            if w.streamed:  # the graph lives in pinned host memory too; its edge blocks are streamed
+                rp_e2e, ci_e2e = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
+            else:
+                rp_e2e, ci_e2e = g.rowptr, g.colidx
+            hplan = B.gnnpre_build_plan(rp_e2e, ci_e2e, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
                                         force_col_slabs=0, segment_edges=args.segment_edges,
-                                        operands_mem=B.GNNPRE_MEM_HOST)
+                                        budget_bytes=int(args.budget_gb * 1e9), operands_mem=B.GNNPRE_MEM_HOST)
             for _ in range(2):
                 B.gnnpre_propagate(hplan, Xh, K, outs_h)
             reps = max(2, min(args.steps, 5))
@@ -304,9 +309,32 @@ def main():
             e2e = {"value": units_per_step / dt, "unit": UNIT, "h2d_bytes_per_step": int(hst.h2d_bytes),
                    "d2h_bytes_per_step": int(hst.d2h_bytes), "ms_per_step": dt * 1e3,
                    "col_slabs": hplan.info()["c"]}
-            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if hplan.info()["c"] == 1 else None
+            hinfo = hplan.info()
+            e2e["blocks"] = hinfo["b"]
+            e2e["structure_on_host"] = bool(hinfo["structure_mem"])
+            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if hinfo["c"] == 1 else None
             e2e["bitwise_equal_to_resident"] = same
+            e2e["max_abs_diff_to_resident"] = max(float((o.cpu() - h).abs().max()) for o, h in zip(outs, outs_h))
             hplan.close()
+            # host-link ceiling measured in this process: one 1 GiB pinned copy per direction, best of 3
+            pin = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+            devb = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+            link = {}
+            for name, dst, src in (("h2d_gbs", devb, pin), ("d2h_gbs", pin, devb)):
+                best = 0.0
+                for _ in range(3):
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                    dst.copy_(src, non_blocking=True)
+                    torch.cuda.synchronize()
+                    best = max(best, (1 << 30) / (time.perf_counter() - t0) / 1e9)
+                link[name] = best
+            moved = max(hst.h2d_bytes, hst.d2h_bytes)
+            link["achieved_gbs"] = moved / dt / 1e9
+            link["direction"] = "d2h" if hst.d2h_bytes >= hst.h2d_bytes else "h2d"
+            link["frac"] = link["achieved_gbs"] / link[link["direction"] + "_gbs"]
+            e2e["host_link"] = link
+            del pin, devb
         except B.GnnpreError as err:
             e2e = {"value": None, "unit": UNIT, "error": str(err)}
 

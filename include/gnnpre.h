@@ -80,7 +80,8 @@ typedef struct {
     int32_t force_col_slabs; /* c; 0 = solve Eq. 12 */
     int32_t segment_edges;   /* edges per warp-level segment; 0 = chosen from F */
     int32_t operands_mem;    /* gnnpre_mem_t: where X and out[] will live at propagate time; HOST makes
-                                Eq. 12 count the library's four slab buffers (beta_X = 4) instead of two */
+                                Eq. 12 count the library's four slab buffers (beta_X = 4) instead of two, and
+                                raises an unforced c = 1 to c = 2 when F >= 128 so that copies and kernels overlap */
     uint32_t flags;
 } gnnpre_plan_opts_t;
 

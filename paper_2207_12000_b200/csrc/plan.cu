@@ -572,6 +572,12 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
         if (!found) return GNNPRE_ERR_BUDGET_TOO_SMALL;
         b = sb;
         c = sc;
+        // Host-resident operands: Eq. 12's model charges every block product the same, but with copies
+        // overlapped a second slab lets the upload of X and the first hop's kernels run side by side.
+        // Two slabs are used when the budget alone asks for one and the row pieces stay >= 256 bytes
+        // (narrower strided pieces travel the host link below full speed).
+        if (opts->force_col_slabs == 0 && opts->operands_mem == GNNPRE_MEM_HOST && c == 1 && F >= 128 && F % 8 == 0)
+            c = 2;
     }
     if (m == 0) b = 1;
     P->b = (int32_t)b;

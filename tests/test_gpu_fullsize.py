@@ -1,0 +1,90 @@
+"""Full-size GPU parity: configuration 4 as bench.py times it, and a scaled configuration 5 streamed
+from pinned host memory with edge blocks and column slabs chosen by the budget solver."""
+import numpy as np
+import pytest
+import torch
+
+import gnnpre_inputs as gi
+import oracle as orc
+from parity_util import TOL, backward_error, hop_error, to_np
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2207_12000_b200 import binding
+    return binding
+
+
+def test_config4_full_size_as_benchmarked(B):
+    """2,449,029 nodes, 123.7M nnz, F=100, K=3, SAGE, 32 blocks, one launch per hop (bench.py's set-up).
+    Integer plan outputs bit-exact; every hop against the full fp64 chain; sampled rows (random, the
+    highest degrees, every block-boundary row) against the exact one-hop result of the matrix the hop
+    read; the degree-weighted column sums SAGE conserves on a symmetric graph."""
+    w = gi.WORKLOADS["c4"]
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    assert (g.n, g.nnz) == (2449029, 123718280)
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, w.feat_dim, force_blocks=w.blocks, force_col_slabs=1)
+    outs, _ = B.gnnpre_propagate(plan, X, w.hops)
+    torch.cuda.synchronize()
+    rp, ci = to_np(g.rowptr), to_np(g.colidx)
+    deg, _, _ = B.gnnpre_plan_scales(plan)
+    np.testing.assert_array_equal(deg.numpy(), orc.degrees(rp))
+    e_off = orc.block_offsets(g.nnz, w.blocks)
+    boundary = []
+    for l in range(w.blocks):
+        blk = B.gnnpre_plan_block(plan, l)
+        assert (blk["e_lo"], blk["e_hi"]) == (e_off[l], e_off[l + 1])
+        assert blk["row_lo"] == np.searchsorted(rp, e_off[l], side="right") - 1
+        boundary += [blk["row_lo"], blk["row_hi"]]
+    d = torch.from_numpy(deg.numpy()).cuda().double()
+    rng = np.random.default_rng(4)
+    rows = np.unique(np.concatenate([rng.integers(0, g.n, 4096), np.argsort(deg.numpy())[-64:], boundary]))
+    want = orc.propagate(w.op, 0.0, rp, ci, to_np(X), w.hops)
+    prev = X
+    for k in range(w.hops):
+        got = to_np(outs[k])
+        assert hop_error(got, want[k]) <= TOL
+        assert backward_error(w.op, 0.0, rp, ci, to_np(prev), got, rows) <= TOL
+        a, b_ = d @ outs[k].double(), d @ prev.double()
+        scale = d @ prev.double().abs()
+        assert float(((a - b_).abs() / scale).max()) <= 1e-6
+        prev = outs[k]
+    plan.close()
+
+
+def test_config5_scaled_streamed_with_budget(B):
+    """Configuration 5 at 1/64 scale (1.7M nodes, 25M nnz, F=128, K=2, GCN): graph, features and outputs in
+    pinned host memory, a budget small enough to force several edge blocks and column slabs."""
+    w = gi.scaled(gi.WORKLOADS["c5"], 64)
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    F, K = w.feat_dim, w.hops
+    rp_h, ci_h = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
+    m = g.nnz + g.n
+    B_S, B_X, B_fixed = 4 * m + 8 * (g.n + 1), 4 * g.n * F, 16 * g.n
+    budget = B_fixed + B_S // 2 + B_X  # room for a quarter of the slab buffers and a quarter of E twice over
+    plan = B.gnnpre_build_plan(rp_h, ci_h, w.op, F, budget_bytes=budget, operands_mem=B.GNNPRE_MEM_HOST)
+    info = plan.info()
+    assert (info["b"], info["c"]) == orc.solve_budget(B_S, B_X, B_fixed, 2, 4, budget, 1 << 20, F // 4)
+    assert info["b"] > 1 and info["c"] > 1 and info["structure_mem"] == 1
+    Xh = X.cpu().pin_memory()
+    outs = [torch.empty((g.n, F), dtype=torch.float32).pin_memory() for _ in range(K)]
+    _, st = B.gnnpre_propagate(plan, Xh, K, outs, want_stats=True)
+    assert st.d2h_bytes == 4 * g.n * F * K
+    assert st.h2d_bytes >= 4 * g.n * F + 4 * m  # X once, and E at least once
+    ref_plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, force_blocks=info["b"], force_col_slabs=info["c"],
+                                   segment_edges=info["segment_edges"])
+    ref, _ = B.gnnpre_propagate(ref_plan, X, K)
+    torch.cuda.synchronize()
+    for k in range(K):
+        assert torch.equal(ref[k].cpu(), outs[k])
+    want = orc.propagate(w.op, 0.0, rp_h.numpy(), ci_h.numpy(), Xh.numpy(), K)
+    for k in range(K):
+        assert hop_error(outs[k].numpy(), want[k]) <= TOL
+    plan.close()
+    ref_plan.close()
