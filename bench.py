@@ -216,6 +216,7 @@ def main():
     g = gi.make_graph(w, device="cuda")
     X = gi.make_features(w, device="cuda")
     torch.cuda.synchronize()
+    torch.cuda.empty_cache()  # the generator's temporaries go back to the driver: the library allocates with cudaMalloc
     gen_s = time.perf_counter() - t0
     K, F = w.hops, w.feat_dim
     blocks = w.blocks if args.blocks < 0 else args.blocks

@@ -67,7 +67,7 @@ def test_config5_scaled_streamed_with_budget(B):
     rp_h, ci_h = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
     m = g.nnz + g.n
     B_S, B_X, B_fixed = 4 * m + 8 * (g.n + 1), 4 * g.n * F, 16 * g.n
-    budget = B_fixed + B_S // 2 + B_X  # room for a quarter of the slab buffers and a quarter of E twice over
+    budget = B_fixed + B_S // 2 + B_X // 8  # far too small for X or E whole: several blocks and many slabs
     plan = B.gnnpre_build_plan(rp_h, ci_h, w.op, F, budget_bytes=budget, operands_mem=B.GNNPRE_MEM_HOST)
     info = plan.info()
     assert (info["b"], info["c"]) == orc.solve_budget(B_S, B_X, B_fixed, 2, 4, budget, 1 << 20, F // 4)
