@@ -81,7 +81,8 @@ typedef struct {
     int32_t segment_edges;   /* edges per warp-level segment; 0 = chosen from F */
     int32_t operands_mem;    /* gnnpre_mem_t: where X and out[] will live at propagate time; HOST makes
                                 Eq. 12 count the library's four slab buffers (beta_X = 4) instead of two, and
-                                raises an unforced c = 1 to c = 2 when F >= 128 so that copies and kernels overlap */
+                                raises an unforced c = 1 to c = 2 (F >= 128) and an unforced b = 1 to b = 8
+                                (|E| >= 2^20) so that copies and kernels overlap */
     uint32_t flags;
 } gnnpre_plan_opts_t;
 

@@ -578,6 +578,9 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
         // (narrower strided pieces travel the host link below full speed).
         if (opts->force_col_slabs == 0 && opts->operands_mem == GNNPRE_MEM_HOST && c == 1 && F >= 128 && F % 8 == 0)
             c = 2;
+        // Likewise a single edge block would hold every output row back until the whole hop is done;
+        // eight blocks let finished rows leave for the host while the rest of the hop computes.
+        if (opts->force_blocks == 0 && opts->operands_mem == GNNPRE_MEM_HOST && b == 1 && m >= (1 << 20)) b = 8;
     }
     if (m == 0) b = 1;
     P->b = (int32_t)b;
