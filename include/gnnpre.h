@@ -103,7 +103,8 @@ typedef struct {
     int64_t num_row_fixups;    /* rows whose edges span more than one segment */
     int64_t num_scratch_rows;  /* partial-sum rows of scratch memory (slab_width floats each) */
     int32_t segment_edges;
-    int32_t structure_mem;     /* gnnpre_mem_t: where the plan's copy of E lives */
+    int32_t structure_mem;     /* gnnpre_mem_t: where the plan's copy of E lives: on the host (streamed block by
+                                  block) only if the CSR was given on the host and b > 1 was forced or needed */
 } gnnpre_plan_info_t;
 
 /* One edge block E^(l): edges [e_lo, e_hi) of the CSR-ordered edge list of the support. */

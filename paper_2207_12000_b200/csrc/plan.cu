@@ -580,7 +580,11 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
             c = 2;
         // Likewise a single edge block would hold every output row back until the whole hop is done;
         // eight blocks let finished rows leave for the host while the rest of the hop computes.
-        if (opts->force_blocks == 0 && opts->operands_mem == GNNPRE_MEM_HOST && b == 1 && m >= (1 << 20)) b = 8;
+        if (opts->force_blocks == 0 && b == 1) {
+            // E fits the budget whole: it stays on the device even when the caller's CSR lives on the host
+            P->structure_mem = GNNPRE_MEM_DEVICE;
+            if (opts->operands_mem == GNNPRE_MEM_HOST && m >= (1 << 20)) b = 8;
+        }
     }
     if (m == 0) b = 1;
     P->b = (int32_t)b;
