@@ -44,6 +44,9 @@ def parse():
     ap.add_argument("--segment-edges", type=int, default=0)
     ap.add_argument("--blocks", type=int, default=-1, help="override the workload's block count")
     ap.add_argument("--per-block-launch", action="store_true")
+    ap.add_argument("--no-bulk-copy", action="store_true", help="register-gather kernel for every width")
+    ap.add_argument("--feat-dim", type=int, default=0, help="override the workload's F (sweeps)")
+    ap.add_argument("--op", type=int, default=-1, help="override the workload's operator (sweeps)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--budget-gb", type=float, default=0.0, help="device-memory budget B_GPU of the streamed plan (0 = free memory)")
     ap.add_argument("--no-e2e", action="store_true")
@@ -192,6 +195,9 @@ def workload_config(w, g, info):
 def main():
     args = parse()
     w = gi.scaled(gi.WORKLOADS[args.workload], args.scale_down)
+    if args.feat_dim or args.op >= 0:
+        import dataclasses
+        w = dataclasses.replace(w, feat_dim=args.feat_dim or w.feat_dim, op=args.op if args.op >= 0 else w.op)
     if args.impl == "reference":
         run_reference(args, w)
         return
@@ -221,6 +227,8 @@ def main():
     K, F = w.hops, w.feat_dim
     blocks = w.blocks if args.blocks < 0 else args.blocks
     flags = B.GNNPRE_FLAG_LAUNCH_PER_BLOCK if args.per_block_launch else 0
+    if args.no_bulk_copy:
+        flags |= B.GNNPRE_FLAG_NO_BULK_COPY
 
     t0 = time.perf_counter()
     plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
@@ -272,7 +280,8 @@ def main():
     launches_per_hop = seg_launches / (args.steps * K)
     seg_launch_ms = seg_ms / max(1, seg_launches)
     achieved = gather_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9
-    traffic = profiled_traffic(w.name) if args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1 else None
+    traffic = (profiled_traffic(w.name) if args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1
+               and not args.no_bulk_copy and not args.feat_dim and args.op < 0 else None)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": traffic,
                 "dram_achieved": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9,

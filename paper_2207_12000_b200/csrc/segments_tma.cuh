@@ -31,7 +31,11 @@ constexpr int kTmaRows = GNNPRE_TMA_ROWS;      // rows per stage = edges per chu
 constexpr int kTmaStep = 8;                    // edges per plain-sum step (same as k_segments' U for G = 32, V = 1)
 constexpr int kTmaMaxWarps = GNNPRE_TMA_WARPS;
 static_assert(kTmaRows % kTmaStep == 0 && kTmaRows <= 32, "a chunk is a whole number of steps and fits one warp");
-constexpr uint32_t kTmaSpinLimit = 1u << 22;
+// A poll that finds the phase incomplete lets the hardware park the warp for up to kTmaSuspendNs
+// before it returns, so waiting warps do not eat the issue slots of working ones; kTmaSpinLimit such
+// polls (about two seconds at most) and the wait gives up.
+constexpr uint32_t kTmaSuspendNs = 20000;
+constexpr uint32_t kTmaSpinLimit = 100000;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -50,10 +54,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t done;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done)
-        : "r"(bar), "r"(parity)
+        : "r"(bar), "r"(parity), "r"(kTmaSuspendNs)
         : "memory");
     return done != 0;
 }
