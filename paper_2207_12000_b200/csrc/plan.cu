@@ -346,8 +346,12 @@ int32_t auto_segment_edges(int64_t slab_width, int64_t m, bool bulk_copy, int nu
         while ((int64_t)p * 2 <= per_warp && p < 4096) p *= 2;
         return p;
     }
-    // about 32 Ki gathered floats per segment, a power of two between 32 and 4096 edges
-    int64_t L = 32768 / std::max<int64_t>(slab_width, 4);
+    // about 32 Ki gathered floats per segment, but short enough that every SM's 2048 threads get a
+    // segment per lane group; a power of two between 32 and 4096 edges
+    const int64_t f4 = std::min<int64_t>(std::max<int64_t>(slab_width, 4), 512) / 4;
+    const int64_t lanes = f4 <= 4 ? 4 : f4 <= 8 ? 8 : f4 <= 16 ? 16 : 32;
+    const int64_t groups = (int64_t)std::max(num_sms, 1) * (2048 / lanes);
+    const int64_t L = std::min<int64_t>(32768 / std::max<int64_t>(slab_width, 4), m / groups);
     int32_t p = 32;
     while ((int64_t)p * 2 <= L && p < 4096) p *= 2;
     return p;
