@@ -596,9 +596,14 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     P->slab_width = 4 * ((F + 4 * c - 1) / (4 * c));
     if (P->slab_width * (c - 1) >= F) return GNNPRE_ERR_INVALID_ARG;  // a slab would be empty
     GNNPRE_CUDA(cudaDeviceGetAttribute(&P->num_sms, cudaDevAttrMultiProcessorCount, P->device));
+    // edges one launch covers: a hop when everything is resident, one block when blocks are launched singly
+    const bool per_block = (opts->flags & GNNPRE_FLAG_LAUNCH_PER_BLOCK) || opts->operands_mem == GNNPRE_MEM_HOST ||
+                           P->structure_mem == GNNPRE_MEM_HOST;
+    const int64_t m_launch = per_block ? m / b : m;
     P->segment_edges = opts->segment_edges > 0
                            ? opts->segment_edges
-                           : auto_segment_edges(P->slab_width, m, uses_bulk_copy(P, (int32_t)P->slab_width), P->num_sms);
+                           : auto_segment_edges(P->slab_width, m_launch, uses_bulk_copy(P, (int32_t)P->slab_width),
+                                                P->num_sms);
     if (P->segment_edges < 1) return GNNPRE_ERR_INVALID_ARG;
 
     // ---- block table: block l = edges [floor(l m / b), floor((l+1) m / b))

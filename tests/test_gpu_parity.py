@@ -327,7 +327,7 @@ def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
     g = gi.rmat(30000, 400000, 17, directed_candidates=True)
     drp, dci = dev(g)
     X = gi.normal_matrix(g.n, F, 9, device="cuda")
-    for b, seg in ((1, 0), (3, 64), (2, 1000)):
+    for b, seg in ((1, 256), (3, 64), (2, 1000)):  # same segment length for both: same summation order
         res = []
         for flags in (0, B.GNNPRE_FLAG_NO_BULK_COPY):
             plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, segment_edges=seg, flags=flags)
