@@ -12,6 +12,8 @@
 // boundary leave their partial sums in scratch rows, which k_row_fixups adds up in a fixed order.
 #include <algorithm>
 
+#include <cuda.h>
+
 #include "gnnpre_internal.cuh"
 
 namespace gnnpre {
@@ -310,20 +312,52 @@ int launch_segments_shape(const gnnpre_plan* P, const SegArgs& a, cudaStream_t s
 // into the SM's shared memory (at most 8).
 constexpr size_t kTmaSmemBudget = 227 * 1024 - 1024;
 
+uint32_t tma_stage_bytes(int32_t f4) { return (kTmaRows / 4) * ((4u * 16u * (uint32_t)f4 + 127u) & ~127u); }
+
 int tma_warps(int32_t f4) {
-    const size_t per_warp = (size_t)kTmaStages * kTmaRows * 16u * (size_t)f4;
+    const size_t per_warp = (size_t)kTmaStages * tma_stage_bytes(f4);
     return (int)std::min<size_t>(kTmaMaxWarps, kTmaSmemBudget / per_warp);
+}
+
+// Tensor map of the [n, width] fp32 matrix at `x` with row stride ldx: box = one row of `width` columns,
+// no swizzle, no interleave.  The driver entry point is looked up once (no link-time dependency on libcuda).
+int make_row_tensor_map(const float* x, int64_t n, int32_t width, int64_t ldx, CUtensorMap* out) {
+    typedef CUresult (*encode_fn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static encode_fn encode = nullptr;
+    if (!encode) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        GNNPRE_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !fn) return GNNPRE_ERR_CUDA;
+        encode = reinterpret_cast<encode_fn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)width, (cuuint64_t)n};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldx * sizeof(float)};
+    const cuuint32_t box[2] = {(cuuint32_t)width, 1u};
+    const cuuint32_t elem[2] = {1u, 1u};
+    const CUresult r = encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(x), dims, strides, box, elem,
+                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        set_last_cuda_error(cudaErrorInvalidValue, "cuTensorMapEncodeTiled", __FILE__, __LINE__);
+        return GNNPRE_ERR_CUDA;
+    }
+    return GNNPRE_OK;
 }
 
 template <int OP, bool HAS_EMPTY>
 int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int nwarps = tma_warps(a.f4);
-    const size_t smem = (size_t)nwarps * kTmaStages * kTmaRows * 16u * (size_t)a.f4;
+    const size_t smem = (size_t)nwarps * kTmaStages * tma_stage_bytes(a.f4);
+    CUtensorMap tmap;
+    GNNPRE_TRY(make_row_tensor_map(a.x, P->n, 4 * a.f4, a.ldx, &tmap));
     auto kernel = k_segments_tma<OP, HAS_EMPTY>;
     GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t nseg = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)std::min<int64_t>(P->num_sms, (nseg + nwarps - 1) / nwarps);
-    kernel<<<grid, nwarps * 32, smem, st>>>(a, P->dev_error.p);
+    kernel<<<grid, nwarps * 32, smem, st>>>(a, tmap, P->dev_error.p);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }

@@ -13,6 +13,14 @@
 // (plain sums over steps of 8 edges, folded into the row's compensated sum): both kernels produce
 // identical bits.
 //
+// Rows travel four at a time: one tile::gather4 tensor copy takes a column offset and four row
+// indices of the [n, width] feature matrix (described by a tensor map whose box is one row high) and
+// lands the four rows back to back in shared memory, so the copy engine is handed one instruction
+// per four edges instead of one per edge (a plain cp.async.bulk per row was measured first: the
+// engine is fed by one lane at a time, smsp__inst_executed_op_tma_ld equalled the edge count, and
+// the issue loop dominated the instruction stream).  Groups of four rows start on 128-byte
+// boundaries, as tensor copies require.
+//
 // Every wait on an mbarrier is bounded: after kTmaSpinLimit polls the warp records an error in
 // a.error, drains what it has in flight (bounded as well) and leaves.
 #pragma once
@@ -30,7 +38,7 @@ constexpr int kTmaStages = GNNPRE_TMA_STAGES;  // chunks a warp keeps in flight
 constexpr int kTmaRows = GNNPRE_TMA_ROWS;      // rows per stage = edges per chunk (8, 16 or 32)
 constexpr int kTmaStep = 8;                    // edges per plain-sum step (same as k_segments' U for G = 32, V = 1)
 constexpr int kTmaMaxWarps = GNNPRE_TMA_WARPS;
-static_assert(kTmaRows % kTmaStep == 0 && kTmaRows <= 32, "a chunk is a whole number of steps and fits one warp");
+static_assert(kTmaRows % kTmaStep == 0 && kTmaRows % 4 == 0 && kTmaRows <= 32, "a chunk is a whole number of steps and fits one warp");
 // A poll that finds the phase incomplete lets the hardware park the warp for up to kTmaSuspendNs
 // before it returns, so waiting warps do not eat the issue slots of working ones; kTmaSpinLimit such
 // polls (about two seconds at most) and the wait gives up.
@@ -69,11 +77,15 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     return false;
 }
 
-// bytes: a multiple of 16; dst (shared) and src (global) 16-byte aligned
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// Four rows r0..r3 of the tensor described by `tmap` (box = [width, 1]), columns from x0 on, land at
+// dst, dst + row bytes, ...  dst is 128-byte aligned, x0 * 4 a multiple of 16.
+__device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tmap, int x0, int r0, int r1, int r2, int r3,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
+        : "memory");
 }
 
 // Per-stage bookkeeping a warp keeps in registers between issuing a chunk and summing it.
@@ -86,14 +98,16 @@ struct TmaChunk {
 };
 
 template <int OP, bool HAS_EMPTY>
-__global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const SegArgs a, int* error) {
+__global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
+    k_segments_tma(const SegArgs a, const __grid_constant__ CUtensorMap tmap, int* error) {
     constexpr unsigned kFull = 0xffffffffu;
     extern __shared__ __align__(128) unsigned char tma_smem[];
     __shared__ __align__(8) unsigned long long bars[kTmaMaxWarps][kTmaStages];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
     const uint32_t rb = 16u * (uint32_t)a.f4;  // bytes of one row of this column tile
-    const uint32_t stage_bytes = kTmaRows * rb;
+    const uint32_t group_bytes = (4u * rb + 127u) & ~127u;  // four rows, padded to the next 128-byte boundary
+    const uint32_t stage_bytes = (kTmaRows / 4) * group_bytes;
     unsigned char* my_smem = tma_smem + (size_t)warp * kTmaStages * stage_bytes;
     const uint32_t smem0 = smem_u32(my_smem);
     const uint32_t bar0 = smem_u32(&bars[warp][0]);
@@ -115,8 +129,6 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
     const bool on = lane < a.f4;  // lanes beyond the row's width re-read column 0 and never store
     const uint32_t lane_off = on ? 16u * lane : 0u;
     const unsigned lt_mask = (1u << lane) - 1u;
-    const uint32_t ldx4 = (uint32_t)(a.ldx >> 2);
-    const float4* xbase = reinterpret_cast<const float4*>(a.x);
 
     const int64_t W = (int64_t)gridDim.x * nwarps;
     for (int64_t s = a.seg_lo + (int64_t)blockIdx.x * nwarps + warp; s < a.seg_hi && !failed; s += W) {
@@ -159,10 +171,15 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
             m.row = row;
             rank_issue += __popc(m.ends);
             const uint32_t bar = bar0 + 8u * st;
-            if (lane == 0) mbar_arrive_expect_tx(bar, (uint32_t)m.cnt * rb);
+            // lanes 0, 4, 8, ... each hand the engine the rows of their four edges (padding lanes hold row 0)
+            const int r0 = (int)(c & ~kRowEndBit);
+            const int r1 = __shfl_down_sync(kFull, r0, 1), r2 = __shfl_down_sync(kFull, r0, 2),
+                      r3 = __shfl_down_sync(kFull, r0, 3);
+            const uint32_t groups = (uint32_t)(m.cnt + 3) >> 2;
+            if (lane == 0) mbar_arrive_expect_tx(bar, groups * 4u * rb);
             __syncwarp();
-            if (lane < m.cnt)
-                bulk_copy_g2s(smem0 + st * stage_bytes + lane * rb, xbase + (uint64_t)(c & ~kRowEndBit) * ldx4, rb, bar);
+            if ((lane & 3) == 0 && lane < m.cnt)
+                tma_gather4(smem0 + st * stage_bytes + (uint32_t)(lane >> 2) * group_bytes, &tmap, 0, r0, r1, r2, r3, bar);
             inflight[st] = true;
         };
 
@@ -202,7 +219,8 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1) k_segments_tma(const Seg
             for (int t0 = 0; t0 < m.cnt; t0 += kTmaStep) {
                 float4 x[kTmaStep];
 #pragma unroll
-                for (int u = 0; u < kTmaStep; ++u) x[u] = *reinterpret_cast<const float4*>(base + (t0 + u) * rb);
+                for (int u = 0; u < kTmaStep; ++u)
+                    x[u] = *reinterpret_cast<const float4*>(base + ((t0 + u) >> 2) * group_bytes + ((t0 + u) & 3) * rb);
                 const unsigned step_ends = (m.ends >> t0) & ((1u << kTmaStep) - 1u);
                 if (step_ends == 0 && t0 + kTmaStep <= m.cnt) {  // no row ends here: a straight run of adds
 #pragma unroll
