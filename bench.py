@@ -322,7 +322,9 @@ def main():
             hinfo = hplan.info()
             e2e["blocks"] = hinfo["b"]
             e2e["structure_on_host"] = bool(hinfo["structure_mem"])
-            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if hinfo["c"] == 1 else None
+            # same bits are expected only when both plans cut the edge list the same way
+            comparable = hinfo["c"] == 1 and hinfo["segment_edges"] == info["segment_edges"]
+            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if comparable else None
             e2e["bitwise_equal_to_resident"] = same
             e2e["max_abs_diff_to_resident"] = max(float((o.cpu() - h).abs().max()) for o, h in zip(outs, outs_h))
             hplan.close()
