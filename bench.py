@@ -123,6 +123,21 @@ def profiled_traffic(workload_name):
     return int(t.group(1)) if cur.hexdigest() == h.group(1) else None
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: every rank runs an independent replica, the job is as slow as the slowest."""
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def aggregate_throughput(units_per_step: int, steps: int, world: int, total_ms: float) -> float:
+    """Whole-job throughput of `world` replicas (weak scaling: per-GPU work is fixed)."""
+    return world * units_per_step * steps / (total_ms * 1e-3)
+
+
 def byte_model(n, m, F):
     """Algorithmic bytes of one hop.  gather: every neighbour row comes from memory once per edge;
     min: every matrix is touched once."""
@@ -267,12 +282,9 @@ def main():
         barrier()
     step_ms = [a.elapsed_time(b_) for a, b_ in ev]
     total_ms = float(sum(step_ms))
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, "cuda")
     units_per_step = K * m * F
-    value = world * units_per_step * args.steps / (total_ms * 1e-3)
+    value = aggregate_throughput(units_per_step, args.steps, world, total_ms)
 
     # ---------------- roofline of the dominant kernel (the segment kernel: one launch = one hop here)
     peak, peak_kind = measured_peaks()
