@@ -347,19 +347,27 @@ int make_row_tensor_map(const float* x, int64_t n, int32_t width, int64_t ldx, C
     return GNNPRE_OK;
 }
 
-template <int OP, bool HAS_EMPTY>
-int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
+template <int OP, bool HAS_EMPTY, int F4C>
+int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int nwarps = tma_warps(a.f4);
     const size_t smem = (size_t)nwarps * kTmaStages * tma_stage_bytes(a.f4);
     CUtensorMap tmap;
     GNNPRE_TRY(make_row_tensor_map(a.x, P->n, 4 * a.f4, a.ldx, &tmap));
-    auto kernel = k_segments_tma<OP, HAS_EMPTY>;
+    auto kernel = k_segments_tma<OP, HAS_EMPTY, F4C>;
     GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t nseg = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)std::min<int64_t>(P->num_sms, (nseg + nwarps - 1) / nwarps);
     kernel<<<grid, nwarps * 32, smem, st>>>(a, tmap, P->dev_error.p);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
+}
+
+// The two widths of the paper's datasets (F = 100, F = 128) get kernels with the row size compiled in.
+template <int OP, bool HAS_EMPTY>
+int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
+    if (a.f4 == 25) return launch_segments_tma_width<OP, HAS_EMPTY, 25>(P, a, st);
+    if (a.f4 == 32) return launch_segments_tma_width<OP, HAS_EMPTY, 32>(P, a, st);
+    return launch_segments_tma_width<OP, HAS_EMPTY, 0>(P, a, st);
 }
 
 int launch_segments_tma(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {

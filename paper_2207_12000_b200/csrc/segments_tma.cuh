@@ -1,5 +1,5 @@
 // Segment kernel with the gathered rows staged through shared memory by the bulk-copy (TMA) engine.
-// Included by propagate.cu inside its unnamed namespace (uses SegArgs, kahan4, kRowEndBit).
+// Included by propagate.cu inside its unnamed namespace (uses SegArgs, Segment, kRowEndBit).
 //
 // Why: the register kernel k_segments keeps at most (warps per SM) x U rows in flight, bounded by
 // the register file; a gather of 400-512 B rows at random addresses needs ~100 KB in flight per SM
@@ -88,6 +88,46 @@ __device__ __forceinline__ void tma_gather4(uint32_t dst, const CUtensorMap* tma
         : "memory");
 }
 
+// A float4 handled as two packed pairs: Blackwell adds and multiplies two fp32 per instruction
+// (add/fma .f32x2).  Each lane of each pair is an ordinary IEEE operation, so results equal the scalar
+// code's bit for bit.
+struct Quad {
+    float2 lo, hi;
+};
+
+__device__ __forceinline__ Quad quad_zero() { return {make_float2(0.f, 0.f), make_float2(0.f, 0.f)}; }
+
+__device__ __forceinline__ Quad quad_load(const unsigned char* p) {
+    const float4 v = *reinterpret_cast<const float4*>(p);
+    return {make_float2(v.x, v.y), make_float2(v.z, v.w)};
+}
+
+__device__ __forceinline__ void quad_add(Quad& a, const Quad& x) {
+    a.lo = __fadd2_rn(a.lo, x.lo);
+    a.hi = __fadd2_rn(a.hi, x.hi);
+}
+
+__device__ __forceinline__ void quad_fma(Quad& a, float w, const Quad& x) {
+    const float2 ww = make_float2(w, w);
+    a.lo = __ffma2_rn(ww, x.lo, a.lo);
+    a.hi = __ffma2_rn(ww, x.hi, a.hi);
+}
+
+// Compensated addition of x into (sum, comp), as kahan1 does per component: a - b is evaluated as
+// fma(-1, b, a), which rounds the same.
+__device__ __forceinline__ void kahan_pair(float2& sum, float2& comp, const float2& x) {
+    const float2 neg = make_float2(-1.f, -1.f);
+    const float2 y = __ffma2_rn(neg, comp, x);
+    const float2 t = __fadd2_rn(sum, y);
+    comp = __ffma2_rn(neg, y, __ffma2_rn(neg, sum, t));
+    sum = t;
+}
+
+__device__ __forceinline__ void quad_kahan(Quad& sum, Quad& comp, const Quad& x) {
+    kahan_pair(sum.lo, comp.lo, x.lo);
+    kahan_pair(sum.hi, comp.hi, x.hi);
+}
+
 // Per-stage bookkeeping a warp keeps in registers between issuing a chunk and summing it.
 struct TmaChunk {
     uint32_t c;      // this lane's column entry (row-end mark in bit 31); 0 on padding lanes
@@ -97,7 +137,8 @@ struct TmaChunk {
     float r, w;      // row scale of that row; weight of this lane's edge
 };
 
-template <int OP, bool HAS_EMPTY>
+// F4C: the row width in float4 when known at compile time (shared-memory offsets become immediates), else 0.
+template <int OP, bool HAS_EMPTY, int F4C>
 __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
     k_segments_tma(const SegArgs a, const __grid_constant__ CUtensorMap tmap, int* error) {
     constexpr unsigned kFull = 0xffffffffu;
@@ -105,7 +146,7 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
     __shared__ __align__(8) unsigned long long bars[kTmaMaxWarps][kTmaStages];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int nwarps = blockDim.x >> 5;
-    const uint32_t rb = 16u * (uint32_t)a.f4;  // bytes of one row of this column tile
+    const uint32_t rb = F4C ? 16u * F4C : 16u * (uint32_t)a.f4;  // bytes of one row of this column tile
     const uint32_t group_bytes = (4u * rb + 127u) & ~127u;  // four rows, padded to the next 128-byte boundary
     const uint32_t stage_bytes = (kTmaRows / 4) * group_bytes;
     unsigned char* my_smem = tma_smem + (size_t)warp * kTmaStages * stage_bytes;
@@ -142,7 +183,7 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
         const int slot_head = g.slot_head, slot_tail = g.slot_tail;
         bool head_pending = slot_head >= 0;
         bool open = false;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f), tot = acc, cmp = acc;
+        Quad acc = quad_zero(), tot = quad_zero(), cmp = quad_zero();
         TmaChunk ch[kTmaStages];
 
         // ---- ask the copy engine for the rows of chunk k, into stage st
@@ -197,13 +238,11 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
                 dst = a.out + (int64_t)row * a.ldo;
                 scale = r;
             }
-            kahan4(tot, cmp, acc);
-            if (on) {
-                float4 o = tot;
-                o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
-                reinterpret_cast<float4*>(dst)[lane] = o;
-            }
-            acc = tot = cmp = make_float4(0.f, 0.f, 0.f, 0.f);
+            quad_kahan(tot, cmp, acc);
+            if (on)
+                reinterpret_cast<float4*>(dst)[lane] =
+                    make_float4(tot.lo.x * scale, tot.lo.y * scale, tot.hi.x * scale, tot.hi.y * scale);
+            acc = tot = cmp = quad_zero();
         };
 
         // ---- sum the rows of the chunk held by stage st
@@ -217,40 +256,30 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
             inflight[st] = false;
             const unsigned char* base = my_smem + st * stage_bytes + lane_off;
             for (int t0 = 0; t0 < m.cnt; t0 += kTmaStep) {
-                float4 x[kTmaStep];
+                Quad x[kTmaStep];
 #pragma unroll
                 for (int u = 0; u < kTmaStep; ++u)
-                    x[u] = *reinterpret_cast<const float4*>(base + ((t0 + u) >> 2) * group_bytes + ((t0 + u) & 3) * rb);
+                    x[u] = quad_load(base + ((t0 + u) >> 2) * group_bytes + ((t0 + u) & 3) * rb);
                 const unsigned step_ends = (m.ends >> t0) & ((1u << kTmaStep) - 1u);
                 if (step_ends == 0 && t0 + kTmaStep <= m.cnt) {  // no row ends here: a straight run of adds
 #pragma unroll
                     for (int u = 0; u < kTmaStep; ++u) {
-                        if (OP == GNNPRE_OP_SAGE_MEAN) {
-                            acc.x += x[u].x; acc.y += x[u].y; acc.z += x[u].z; acc.w += x[u].w;
-                        } else {
-                            const float ww = __shfl_sync(kFull, m.w, t0 + u);
-                            acc.x = fmaf(ww, x[u].x, acc.x); acc.y = fmaf(ww, x[u].y, acc.y);
-                            acc.z = fmaf(ww, x[u].z, acc.z); acc.w = fmaf(ww, x[u].w, acc.w);
-                        }
+                        if (OP == GNNPRE_OP_SAGE_MEAN) quad_add(acc, x[u]);
+                        else quad_fma(acc, __shfl_sync(kFull, m.w, t0 + u), x[u]);
                     }
                 } else {
 #pragma unroll
                     for (int u = 0; u < kTmaStep; ++u) {
                         const int t = t0 + u;
                         if (t < m.cnt) {
-                            if (OP == GNNPRE_OP_SAGE_MEAN) {
-                                acc.x += x[u].x; acc.y += x[u].y; acc.z += x[u].z; acc.w += x[u].w;
-                            } else {
-                                const float ww = __shfl_sync(kFull, m.w, t);
-                                acc.x = fmaf(ww, x[u].x, acc.x); acc.y = fmaf(ww, x[u].y, acc.y);
-                                acc.z = fmaf(ww, x[u].z, acc.z); acc.w = fmaf(ww, x[u].w, acc.w);
-                            }
+                            if (OP == GNNPRE_OP_SAGE_MEAN) quad_add(acc, x[u]);
+                            else quad_fma(acc, __shfl_sync(kFull, m.w, t), x[u]);
                             if ((m.ends >> t) & 1u) flush(t, m);
                         }
                     }
                 }
-                kahan4(tot, cmp, acc);  // this step's plain sum joins the row's compensated sum
-                acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                quad_kahan(tot, cmp, acc);  // this step's plain sum joins the row's compensated sum
+                acc = quad_zero();
             }
             open = ((m.ends >> (m.cnt - 1)) & 1u) == 0;
             __syncwarp();  // every lane is done with the stage before it is refilled
@@ -273,7 +302,8 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
         if (open) {  // the row holding the last edge continues in the next segment
             const int slot = head_pending ? slot_head : slot_tail;
             if (slot >= 0 && on)
-                reinterpret_cast<float4*>(a.scratch + (int64_t)slot * a.scratch_ld)[lane] = tot;
+                reinterpret_cast<float4*>(a.scratch + (int64_t)slot * a.scratch_ld)[lane] =
+                    make_float4(tot.lo.x, tot.lo.y, tot.hi.x, tot.hi.y);
         }
     }
 
