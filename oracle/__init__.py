@@ -57,6 +57,7 @@ def _c():
         lib.orc_solve_budget.restype = ctypes.c_int
         lib.orc_solve_normalisation_blocks.argtypes = [i64] * 8
         lib.orc_solve_normalisation_blocks.restype = i64
+        lib.orc_normalized_values.argtypes = [ctypes.c_int, f64, i64, p, p, p]
         lib.orc_slab_width.argtypes = [i64, i64]
         lib.orc_slab_width.restype = i64
         lib.orc_propagate_blocked.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, ctypes.c_int, i32, i32, p]
@@ -181,6 +182,14 @@ def solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
 
 def solve_normalisation_blocks(B_A, B_S, B_D, alpha_A, alpha_S, alpha_D, B_GPU, max_a):
     return int(_c().orc_solve_normalisation_blocks(B_A, B_S, B_D, alpha_A, alpha_S, alpha_D, B_GPU, max_a))
+
+
+def normalized_values(op: int, eps: float, rowptr, colidx) -> np.ndarray:
+    """fp64 value of every edge of the support, in the order of support(op, rowptr, colidx)."""
+    rowptr, colidx, n = _csr(rowptr, colidx)
+    vals = np.empty(support_nnz(op, n, int(rowptr[n])), dtype=np.float64)
+    _c().orc_normalized_values(op, float(eps), n, _ptr(rowptr), _ptr(colidx), _ptr(vals))
+    return vals
 
 
 def slab_width(F: int, c: int) -> int:

@@ -295,6 +295,34 @@ int64_t orc_solve_normalisation_blocks(int64_t B_A, int64_t B_S, int64_t B_D, in
     return -1;
 }
 
+/*
+ * The normalised adjacency itself (Eq. 1; block-wise Eq. 10): the value A^_ij of every edge of the
+ * support, in the support's CSR order (orc_support gives the matching structure).  With b blocks,
+ * block l holds the values of edges [e_off[l], e_off[l+1]); the blocks are disjoint, so their
+ * union is the whole matrix.  vals has orc_support_nnz entries.
+ */
+void orc_normalized_values(int op, double eps, int64_t n, const int64_t* rowptr, const int32_t* colidx, double* vals) {
+    int32_t* deg = (int32_t*)malloc(sizeof(int32_t) * (size_t)n);
+    orc_degrees(n, rowptr, deg);
+    int64_t w = 0;
+    for (int64_t i = 0; i < n; ++i) {
+        int64_t e = rowptr[i];
+        const int64_t end = rowptr[i + 1];
+        int diag_pending = has_diagonal(op);
+        while (e < end || diag_pending) {
+            int64_t j;
+            if (diag_pending && (e == end || colidx[e] > i)) {
+                j = i;
+                diag_pending = 0;
+            } else {
+                j = colidx[e++];
+            }
+            vals[w++] = entry(op, eps, deg, i, j);
+        }
+    }
+    free(deg);
+}
+
 /* Width of a column slab: ceil(F / c) rounded up to a multiple of 4 columns. */
 int64_t orc_slab_width(int64_t F, int64_t c) { return 4 * ceil_div(F, 4 * c); }
 

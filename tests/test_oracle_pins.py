@@ -418,3 +418,44 @@ def test_paper_block_counts_are_feasible(golden_dir):
 def test_slab_width():
     assert orc.slab_width(128, 1) == 128 and orc.slab_width(128, 16) == 8
     assert orc.slab_width(100, 3) == 36 and orc.slab_width(10, 2) == 8
+
+
+# ------------------------------------------------------------------ the normalised adjacency itself (Eq. 1 / Eq. 10)
+
+@pytest.mark.parametrize("op", OPS)
+def test_normalized_values_rebuild_the_dense_operator(op):
+    """The per-edge values, scattered by the support's structure, are the dense operator built in this
+    test from its definition; every block of Eq. 10 is a slice of them and the blocks sum to S."""
+    n = 40
+    rowptr, colidx = random_graph(n, 100, 95)
+    A = dense_adjacency(rowptr, colidx)
+    d = A.sum(1)
+    if op == orc.OP_GCN:
+        At = A + np.eye(n)
+        dinv = 1.0 / np.sqrt(At.sum(1))
+        want = dinv[:, None] * At * dinv[None, :]
+    elif op == orc.OP_SAGE:
+        want = np.divide(A, d[:, None], out=np.zeros_like(A), where=d[:, None] > 0)
+    else:
+        want = A + (1 + EPS) * np.eye(n)
+    rp, ci = orc.support(op, rowptr, colidx)
+    vals = orc.normalized_values(op, EPS, rowptr, colidx)
+    assert vals.shape == (rp[-1],)
+    got = sp.csr_matrix((vals, ci, rp), shape=(n, n)).toarray()
+    np.testing.assert_allclose(got, want, rtol=1e-15, atol=0)
+    if op == orc.OP_GCN:
+        np.testing.assert_allclose(got, got.T, rtol=1e-15)
+    if op == orc.OP_SAGE:
+        np.testing.assert_allclose(got.sum(1)[d > 0], 1.0, rtol=1e-14)
+    for b in (1, 3, 7):
+        e = orc.block_offsets(int(rp[-1]), b)
+        total = np.zeros((n, n))
+        rows_of_edge = np.repeat(np.arange(n), np.diff(rp))
+        for l in range(b):
+            blk = np.zeros((n, n))
+            blk[rows_of_edge[e[l]:e[l + 1]], ci[e[l]:e[l + 1]]] = vals[e[l]:e[l + 1]]
+            total += blk
+        np.testing.assert_array_equal(total, got)  # Eq. 10: S = sum_l D~^{-1/2} A~^(l) D~^{-1/2}
+    X = features(n, 3, 96)
+    np.testing.assert_allclose(got @ X.astype(np.float64), orc.propagate(op, EPS, rowptr, colidx, X, 1)[0], rtol=1e-13,
+                               atol=1e-14)
