@@ -178,6 +178,23 @@ int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t*
 int gnnpre_propagate(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t x_mem, int32_t K, float* const* out,
                      int64_t ldo, int32_t out_mem, void* stream, gnnpre_stats_t* stats);
 
+/*
+ * The normalised adjacency itself (Eq. 1), computed block-wise as Eq. 10 states it:
+ * vals_out[e] = A^_ij for every edge e = (i, j) of the support, in the CSR order that
+ * gnnpre_plan_support returns, nnz_tilde fp32 values.  Each value is evaluated in fp64 from the
+ * integer degrees and rounded once.  vals_out lives where vals_mem says.  Device-resident structure and
+ * output: one launch on `stream`, asynchronous.  Otherwise the plan's b edge blocks play the role of
+ * the paper's `a` passes - block E^(l) travels to the device if it lives on the host, its values travel
+ * back if wanted on the host, two buffers taking turns - and the call returns when vals_out is complete
+ * (GNNPRE_ERR_BUSY if a streamed call holds the plan).  gnnpre_propagate never needs this array.
+ */
+int gnnpre_normalize(gnnpre_plan_t* plan, float* vals_out, int32_t vals_mem, void* stream);
+
+/* Eq. 11 on its own: least a with ceil((alpha_A B_A + alpha_S B_S) / a) + alpha_D B_D <= B_GPU, 1 <= a <= max_a;
+ * BUDGET_TOO_SMALL if there is none.  Host only. */
+int gnnpre_solve_normalisation_blocks(int64_t B_A, int64_t B_S, int64_t B_D, int64_t alpha_A, int64_t alpha_S,
+                                      int64_t alpha_D, int64_t B_GPU, int64_t max_a, int64_t* a_out);
+
 void gnnpre_plan_destroy(gnnpre_plan_t* plan);
 
 /*

@@ -83,6 +83,8 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
                                      ctypes.POINTER(gnnpre_stats_t)]
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
+    lib.gnnpre_normalize.argtypes = [p, p, i32, p]
+    lib.gnnpre_solve_normalisation_blocks.argtypes = [i64] * 8 + [ctypes.POINTER(i64)]
     lib.gnnpre_plan_destroy.argtypes = [p]
     lib.gnnpre_plan_destroy.restype = None
     lib.gnnpre_solve_budget.argtypes = [i64] * 8 + [ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -230,6 +232,26 @@ def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: to
     return out
 
 
+def gnnpre_normalize(plan: Plan, out: torch.Tensor | None = None, *, host: bool = False, stream=None) -> torch.Tensor:
+    """fp32 value of every edge of the support (order of gnnpre_plan_support), on the device or in host memory."""
+    m = gnnpre_plan_info(plan)["nnz_tilde"]
+    if out is None:
+        out = torch.empty(m, dtype=torch.float32, pin_memory=True) if host else torch.empty(
+            m, dtype=torch.float32, device="cuda")
+    assert out.dtype == torch.float32 and out.numel() == m and out.is_contiguous()
+    _check(_lib.gnnpre_normalize(plan.handle, out.data_ptr(), _mem_of(out), _stream_ptr(stream)), "gnnpre_normalize")
+    return out
+
+
+def gnnpre_solve_normalisation_blocks(B_A, B_S, B_D, alpha_A, alpha_S, alpha_D, B_GPU, max_a):
+    a = ctypes.c_int64()
+    rc = _lib.gnnpre_solve_normalisation_blocks(B_A, B_S, B_D, alpha_A, alpha_S, alpha_D, B_GPU, max_a, ctypes.byref(a))
+    if rc == -6:
+        return -1
+    _check(rc, "gnnpre_solve_normalisation_blocks")
+    return a.value
+
+
 def gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
     b, c = ctypes.c_int64(), ctypes.c_int64()
     rc = _lib.gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c, ctypes.byref(b),
@@ -246,5 +268,6 @@ def gnnpre_status_string(status: int) -> str:
 
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
-            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_normalize",
+            "gnnpre_solve_normalisation_blocks", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

@@ -6,7 +6,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["plan.cu", "propagate.cu", "stream.cu", "noalloc.cu", "api.cu"]
+SOURCES = ["plan.cu", "propagate.cu", "stream.cu", "noalloc.cu", "normalize.cu", "api.cu"]
 LIB = os.path.join(HERE, "lib", "libgnnpre.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -15,7 +15,8 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 
 def _inputs():
     src = [os.path.join(HERE, "csrc", s) for s in SOURCES]
-    hdr = [os.path.join(HERE, "csrc", "gnnpre_internal.cuh"), os.path.join(ROOT, "include", "gnnpre.h")]
+    hdr = [os.path.join(HERE, "csrc", "gnnpre_internal.cuh"), os.path.join(HERE, "csrc", "segments_tma.cuh"),
+           os.path.join(ROOT, "include", "gnnpre.h")]
     return src, hdr
 
 

@@ -80,3 +80,14 @@ def test_null_and_bad_arguments_fail_without_a_device(binding):
     assert lib.gnnpre_propagate(None, None, 0, 0, 1, None, 0, 0, None, None) == -1
     assert lib.gnnpre_degrees(None, None, None) == -1
     lib.gnnpre_plan_destroy(None)  # no-op
+
+
+def test_normalisation_block_count_matches_oracle(binding):
+    rng = np.random.default_rng(3)
+    for _ in range(300):
+        B_A, B_S, B_D = (int(rng.integers(0, 5000)) for _ in range(3))
+        al = [int(rng.integers(0, 4)) for _ in range(3)]
+        B_GPU = int(rng.integers(1, 6000))
+        want = orc.solve_normalisation_blocks(B_A, B_S, B_D, al[0], al[1], al[2], B_GPU, 64)
+        got = binding.gnnpre_solve_normalisation_blocks(B_A, B_S, B_D, al[0], al[1], al[2], B_GPU, 64)
+        assert got == want, (B_A, B_S, B_D, al, B_GPU)

@@ -337,3 +337,32 @@ def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
         for k in range(2):
             assert torch.equal(res[0][k], res[1][k]), (b, seg, k)
     check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[0])
+
+
+# ------------------------------------------------------------------ the normalised adjacency itself
+
+@pytest.mark.parametrize("op", OPS)
+def test_normalized_adjacency_values_bit_exact(B, op):
+    """gnnpre_normalize against the oracle: fp64 evaluation from integer degrees, one rounding to fp32, so
+    the comparison is bitwise; resident and block-streamed (host CSR, host output) runs give the same array."""
+    for name, g in list(small_graphs()) + [("c1", gi.make_graph(gi.WORKLOADS["c1"]))]:
+        rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+        want = orc.normalized_values(op, EPS, rp, ci).astype(np.float32)
+        if want.size == 0:
+            continue
+        for b in (1, 3):
+            if b > want.size:
+                continue
+            plan = B.gnnpre_build_plan(*dev(g), op, 16, gin_eps=EPS, force_blocks=b)
+            got = B.gnnpre_normalize(plan)
+            torch.cuda.synchronize()
+            np.testing.assert_array_equal(to_np(got).view(np.uint32), want.view(np.uint32), err_msg=f"{name} b={b}")
+            plan.close()
+            hplan = B.gnnpre_build_plan(g.rowptr.pin_memory(), g.colidx.pin_memory(), op, 16, gin_eps=EPS,
+                                        force_blocks=b)
+            assert hplan.info()["structure_mem"] == 1
+            for host_out in (True, False):
+                got = B.gnnpre_normalize(hplan, host=host_out)
+                torch.cuda.synchronize()
+                np.testing.assert_array_equal(to_np(got).view(np.uint32), want.view(np.uint32))
+            hplan.close()
