@@ -195,6 +195,16 @@ int gnnpre_normalize(gnnpre_plan_t* plan, float* vals_out, int32_t vals_mem, voi
 int gnnpre_solve_normalisation_blocks(int64_t B_A, int64_t B_S, int64_t B_D, int64_t alpha_A, int64_t alpha_S,
                                       int64_t alpha_D, int64_t B_GPU, int64_t max_a, int64_t* a_out);
 
+/*
+ * Failure-detection self-test (no counterpart in the paper).  The bulk-copy kernel never waits without
+ * a limit: a wait that runs out sets an error word in the plan and the warp leaves; the next
+ * synchronising call returns GNNPRE_ERR_TIMEOUT and clears the word.  This call exercises exactly that
+ * path without any fault: one warp waits `polls` times (1..100000, each poll parks the warp for up to
+ * 20 us) on a barrier that nothing completes.  Returns GNNPRE_ERR_TIMEOUT when the path works, and
+ * leaves the device and the plan fully usable.  Synchronous.
+ */
+int gnnpre_selftest_wait_timeout(gnnpre_plan_t* plan, uint32_t polls, void* stream);
+
 void gnnpre_plan_destroy(gnnpre_plan_t* plan);
 
 /*

@@ -85,6 +85,7 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
     lib.gnnpre_normalize.argtypes = [p, p, i32, p]
     lib.gnnpre_solve_normalisation_blocks.argtypes = [i64] * 8 + [ctypes.POINTER(i64)]
+    lib.gnnpre_selftest_wait_timeout.argtypes = [p, ctypes.c_uint32, p]
     lib.gnnpre_plan_destroy.argtypes = [p]
     lib.gnnpre_plan_destroy.restype = None
     lib.gnnpre_solve_budget.argtypes = [i64] * 8 + [ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -252,6 +253,11 @@ def gnnpre_solve_normalisation_blocks(B_A, B_S, B_D, alpha_A, alpha_S, alpha_D, 
     return a.value
 
 
+def gnnpre_selftest_wait_timeout(plan: Plan, polls: int = 200, stream=None) -> int:
+    """Status of a device wait that is made to run out (expected: -8, GNNPRE_ERR_TIMEOUT)."""
+    return int(_lib.gnnpre_selftest_wait_timeout(plan.handle, polls, _stream_ptr(stream)))
+
+
 def gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
     b, c = ctypes.c_int64(), ctypes.c_int64()
     rc = _lib.gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c, ctypes.byref(b),
@@ -269,5 +275,5 @@ def gnnpre_status_string(status: int) -> str:
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
             "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_normalize",
-            "gnnpre_solve_normalisation_blocks", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

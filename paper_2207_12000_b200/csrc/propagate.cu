@@ -209,6 +209,19 @@ __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(co
 
 #include "segments_tma.cuh"
 
+// A wait on a barrier that nothing ever completes: the polls run out, the error word is set, the warp
+// leaves.  This is the give-up path of k_segments_tma, exercised on its own.
+__global__ void k_wait_that_runs_out(int* error, uint32_t polls) {
+    __shared__ __align__(8) unsigned long long bar;
+    const uint32_t b = smem_u32(&bar);
+    if (threadIdx.x == 0) mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncwarp();
+    bool done = false;
+    for (uint32_t i = 0; i < polls && !done; ++i) done = mbar_try_wait(b, 0);
+    if (!done && threadIdx.x == 0) atomicExch(error, 1);
+}
+
 struct FixArgs {
     const RowFixup* fix;
     int64_t fix_lo, fix_hi;
@@ -543,3 +556,14 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
 }
 
 }  // namespace gnnpre
+
+// Failure-detection self-test: see include/gnnpre.h.
+extern "C" int gnnpre_selftest_wait_timeout(gnnpre_plan_t* P, uint32_t polls, void* stream) {
+    if (!P || !P->dev_error.p || polls == 0 || polls > 100000u) return GNNPRE_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    gnnpre::k_wait_that_runs_out<<<1, 32, 0, st>>>(P->dev_error.p, polls);
+    GNNPRE_CUDA(cudaGetLastError());
+    GNNPRE_CUDA(cudaStreamSynchronize(st));
+    return gnnpre::check_device_error(P);
+}
+

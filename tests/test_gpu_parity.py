@@ -366,3 +366,18 @@ def test_normalized_adjacency_values_bit_exact(B, op):
                 torch.cuda.synchronize()
                 np.testing.assert_array_equal(to_np(got).view(np.uint32), want.view(np.uint32))
             hplan.close()
+
+
+def test_a_device_wait_that_runs_out_is_reported_and_leaves_the_plan_usable(B):
+    """Failure detection without a fault: a warp polls a barrier that nothing completes, gives up after its
+    limit and sets the plan's error word; the host reads GNNPRE_ERR_TIMEOUT once, and the same plan then
+    propagates correctly."""
+    g = gi.erdos_renyi(3000, 20000, 23)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    plan = B.gnnpre_build_plan(*dev(g), 0, 128)
+    assert B.gnnpre_selftest_wait_timeout(plan, 200) == -8
+    assert B.gnnpre_status_string(-8) == "timed out"
+    X = gi.normal_matrix(g.n, 128, 2, device="cuda")
+    outs, st = B.gnnpre_propagate(plan, X, 2, want_stats=True)  # the error word was cleared: no stale timeout
+    check_all_hops(0, 0.0, rp, ci, to_np(X), outs)
+    plan.close()
