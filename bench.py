@@ -374,6 +374,8 @@ def main():
                 "config": workload_config(w, g, info), "clocks": clocks.summary(), "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "plan_build_ms": plan_ms, "input_generation_s": gen_s,
+                # the same metric if every step also rebuilt the plan (degrees, scales, Eq. 12, edge blocks, segments)
+                "value_including_plan_build": world * units_per_step / ((total_ms / args.steps + plan_ms) * 1e-3),
                 "hop_ms": [float(st.hop_ms[k]) for k in range(K)]}
         print(json.dumps(line), flush=True)
     plan.close()
