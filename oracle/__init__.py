@@ -49,6 +49,7 @@ def _c():
         lib.orc_dense_operator.argtypes = [ctypes.c_int, f64, i64, p, p, p]
         lib.orc_hop_f64.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, p]
         lib.orc_propagate.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, ctypes.c_int, p]
+        lib.orc_propagate_teleport.argtypes = [ctypes.c_int, f64, f64, i64, p, p, i64, p, i64, ctypes.c_int, p]
         lib.orc_hop_rows_f32.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, i64, p, p, p]
         lib.orc_block_offsets.argtypes = [i64, i32, p]
         lib.orc_block_offsets.restype = ctypes.c_int
@@ -141,6 +142,16 @@ def propagate(op: int, eps: float, rowptr, colidx, X, K: int) -> np.ndarray:
     F = X.shape[1]
     out = np.empty((K, n, F), dtype=np.float64)
     _c().orc_propagate(op, float(eps), n, _ptr(rowptr), _ptr(colidx), F, _ptr(X), ldx, K, _ptr(out))
+    return out
+
+
+def propagate_teleport(op: int, eps: float, alpha: float, rowptr, colidx, X, K: int) -> np.ndarray:
+    """[K, n, F] fp64: X_k = (1 - alpha) A^ X_{k-1} + alpha X_0."""
+    rowptr, colidx, n = _csr(rowptr, colidx)
+    X, ldx = _f32_matrix(X)
+    F = X.shape[1]
+    out = np.empty((K, n, F), dtype=np.float64)
+    _c().orc_propagate_teleport(op, float(eps), float(alpha), n, _ptr(rowptr), _ptr(colidx), F, _ptr(X), ldx, K, _ptr(out))
     return out
 
 

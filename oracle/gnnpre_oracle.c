@@ -203,6 +203,22 @@ void orc_propagate(int op, double eps, int64_t n, const int64_t* rowptr, const i
 }
 
 /*
+ * Personalised-PageRank style propagation, one of the constant filters Section 3.1 ("Limitation")
+ * names as precomputable:  X_k = (1 - alpha) A^ X_{k-1} + alpha X_0,  k = 1..K  (the power
+ * iteration of APPNP).  alpha = 0 is orc_propagate.  `out` as in orc_propagate.
+ */
+void orc_propagate_teleport(int op, double eps, double alpha, int64_t n, const int64_t* rowptr, const int32_t* colidx,
+                            int64_t F, const float* X, int64_t ldx, int K, double* out) {
+    orc_propagate(op, eps, n, rowptr, colidx, F, X, ldx, 1, out); /* A^ X_0 */
+    for (int k = 0; k < K; ++k) {
+        double* xk = out + (size_t)k * (size_t)n * (size_t)F;
+        if (k > 0) orc_hop_f64(op, eps, n, rowptr, colidx, F, out + (size_t)(k - 1) * (size_t)n * (size_t)F, xk);
+        for (int64_t i = 0; i < n; ++i)
+            for (int64_t f = 0; f < F; ++f) xk[i * F + f] = (1.0 - alpha) * xk[i * F + f] + alpha * (double)X[i * ldx + f];
+    }
+}
+
+/*
  * One hop evaluated on chosen rows only, from an fp32 previous hop: the exact fp64 value
  * of (A^ xprev)[rows[r], :] and, optionally, of (|A^| |xprev|)[rows[r], :].
  */

@@ -459,3 +459,41 @@ def test_normalized_values_rebuild_the_dense_operator(op):
     X = features(n, 3, 96)
     np.testing.assert_allclose(got @ X.astype(np.float64), orc.propagate(op, EPS, rowptr, colidx, X, 1)[0], rtol=1e-13,
                                atol=1e-14)
+
+
+# ------------------------------------------------------------------ teleport (PPR) filter
+
+@pytest.mark.parametrize("op", OPS)
+def test_teleport_propagation_pins(op):
+    """X_k = (1-a) A^ X_{k-1} + a X_0: a = 0 is the plain chain, a = 1 returns X_0, and for GCN/SAGE the
+    iteration converges to the dense solution a (I - (1-a) A^)^{-1} X_0 (computed here with numpy)."""
+    n, F = 30, 4
+    rowptr, colidx = random_graph(n, 80, 97)
+    X = features(n, F, 97)
+    Xd = X.astype(np.float64)
+    np.testing.assert_array_equal(orc.propagate_teleport(op, EPS, 0.0, rowptr, colidx, X, 3),
+                                  orc.propagate(op, EPS, rowptr, colidx, X, 3))
+    np.testing.assert_array_equal(orc.propagate_teleport(op, EPS, 1.0, rowptr, colidx, X, 3), np.stack([Xd] * 3))
+    a = 0.15
+    got = orc.propagate_teleport(op, EPS, a, rowptr, colidx, X, 3)
+    Ahat = orc.dense_operator(op, EPS, rowptr, colidx)
+    cur = Xd
+    for k in range(3):
+        cur = (1 - a) * (Ahat @ cur) + a * Xd
+        np.testing.assert_allclose(got[k], cur, rtol=1e-13, atol=1e-14)
+    if op != orc.OP_GIN:  # spectral radius <= 1: the iteration contracts with factor 1-a
+        far = orc.propagate_teleport(op, EPS, 0.5, rowptr, colidx, X, 60)[-1]
+        fixed = 0.5 * np.linalg.solve(np.eye(n) - 0.5 * Ahat, Xd)
+        np.testing.assert_allclose(far, fixed, rtol=1e-10, atol=1e-12)
+
+
+def test_teleport_on_complete_graph_closed_form():
+    """K_n under GCN: A^ x = column mean, and the mean is preserved, so X_k = (1-a) mean + a X_0 for every k."""
+    n, F, a = 8, 3, 0.3
+    rowptr, colidx = csr_of(n, list(itertools.combinations(range(n), 2)))
+    X = features(n, F, 98)
+    Xd = X.astype(np.float64)
+    want = (1 - a) * np.tile(Xd.mean(0), (n, 1)) + a * Xd
+    got = orc.propagate_teleport(orc.OP_GCN, 0.0, a, rowptr, colidx, X, 4)
+    for k in range(4):
+        np.testing.assert_allclose(got[k], want, rtol=1e-13, atol=1e-15)
