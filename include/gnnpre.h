@@ -84,6 +84,9 @@ typedef struct {
                                 raises an unforced c = 1 to c = 2 (F >= 128) and an unforced b = 1 to b = 8
                                 (|E| >= 2^20) so that copies and kernels overlap */
     uint32_t flags;
+    float teleport_alpha;    /* 0 = plain propagation X_k = A^ X_{k-1}; in (0, 1]: the personalised-PageRank power
+                                iteration X_k = (1 - alpha) A^ X_{k-1} + alpha X_0, another constant filter that
+                                Section 3.1 ("Limitation") lists as precomputable */
 } gnnpre_plan_opts_t;
 
 typedef struct gnnpre_plan gnnpre_plan_t; /* opaque; owns device (and pinned host) memory */
@@ -159,7 +162,8 @@ int gnnpre_plan_scales(const gnnpre_plan_t* plan, int32_t* deg_out, float* rscal
 int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t* colidx_out);
 
 /*
- * Algorithm 1: out[k-1] <- A^ applied k times to X, for k = 1..K (X itself is not repeated).
+ * Algorithm 1: out[k-1] <- A^ applied k times to X, for k = 1..K (X itself is not repeated); with a
+ * teleport term in the plan, out[k-1] <- (1 - alpha) A^ out[k-2] + alpha X instead.
  *   X      fp32 row-major [n, F] with leading dimension ldx (floats), in x_mem
  *   out    host array of K pointers, each fp32 row-major [n, F] with leading dimension ldo, in out_mem
  *   ldx, ldo >= F and multiples of 4; all base pointers 16-byte aligned (else GNNPRE_ERR_ALIGN)

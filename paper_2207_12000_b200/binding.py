@@ -29,7 +29,8 @@ class gnnpre_plan_opts_t(ctypes.Structure):
     _fields_ = [("op", ctypes.c_int32), ("gin_eps", ctypes.c_float), ("feat_dim", ctypes.c_int64),
                 ("budget_bytes", ctypes.c_int64), ("force_blocks", ctypes.c_int32),
                 ("force_col_slabs", ctypes.c_int32), ("segment_edges", ctypes.c_int32),
-                ("operands_mem", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+                ("operands_mem", ctypes.c_int32), ("flags", ctypes.c_uint32),
+                ("teleport_alpha", ctypes.c_float)]
 
 
 class gnnpre_plan_info_t(ctypes.Structure):
@@ -154,10 +155,11 @@ class Plan:
 
 def gnnpre_build_plan(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, feat_dim: int, *, degrees=None,
                       gin_eps: float = 0.0, budget_bytes: int = 0, force_blocks: int = 0, force_col_slabs: int = 0,
-                      segment_edges: int = 0, operands_mem: int = GNNPRE_MEM_DEVICE, flags: int = 0) -> Plan:
+                      segment_edges: int = 0, operands_mem: int = GNNPRE_MEM_DEVICE, flags: int = 0,
+                      teleport_alpha: float = 0.0) -> Plan:
     csr = _csr(rowptr, colidx)
     opts = gnnpre_plan_opts_t(op, gin_eps, feat_dim, budget_bytes, force_blocks, force_col_slabs, segment_edges,
-                              operands_mem, flags)
+                              operands_mem, flags, teleport_alpha)
     if degrees is not None:
         assert degrees.dtype == torch.int32 and degrees.device == rowptr.device and degrees.is_contiguous()
     out = ctypes.c_void_p()

@@ -126,6 +126,7 @@ struct gnnpre_plan {
     int64_t n = 0, nnz = 0, nnz_tilde = 0, feat_dim = 0;
     int32_t op = 0;
     float gin_eps = 0.f;
+    float teleport_alpha = 0.f;
     int32_t b = 1, c = 1;
     int64_t slab_width = 0;
     int64_t B_S = 0, B_X = 0, B_fixed = 0, beta_S = 1, beta_X = 2, budget_bytes = 0;
@@ -175,6 +176,8 @@ struct HopArgs {
     float* xout;             // [n, ldo], likewise
     int64_t ldo;
     int32_t width;           // columns of this slab (multiple of 4)
+    const float* x0;         // [n, ldx0] the slab of X_0, read only when the plan has a teleport term
+    int64_t ldx0;
 };
 
 // propagate.cu

@@ -440,6 +440,7 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     P->feat_dim = opts->feat_dim;
     P->op = opts->op;
     P->gin_eps = opts->gin_eps;
+    P->teleport_alpha = opts->teleport_alpha;
     P->flags = opts->flags;
     P->structure_mem = csr->mem;
     const int64_t m = P->nnz_tilde;
@@ -744,6 +745,7 @@ extern "C" int gnnpre_build_plan(const gnnpre_csr_t* csr, const int32_t* degrees
     if (csr->mem != GNNPRE_MEM_DEVICE && csr->mem != GNNPRE_MEM_HOST) return GNNPRE_ERR_INVALID_ARG;
     if (opts->op < GNNPRE_OP_GCN_SYM || opts->op > GNNPRE_OP_GIN_SUM) return GNNPRE_ERR_INVALID_ARG;
     if (opts->operands_mem != GNNPRE_MEM_DEVICE && opts->operands_mem != GNNPRE_MEM_HOST) return GNNPRE_ERR_INVALID_ARG;
+    if (!(opts->teleport_alpha >= 0.f && opts->teleport_alpha <= 1.f)) return GNNPRE_ERR_INVALID_ARG;
     if (opts->feat_dim < 4) return GNNPRE_ERR_INVALID_ARG;
     if (opts->feat_dim % 4 != 0) return GNNPRE_ERR_ALIGN;
     if (opts->segment_edges < 0 || opts->segment_edges > (1 << 20)) return GNNPRE_ERR_INVALID_ARG;

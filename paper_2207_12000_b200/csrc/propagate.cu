@@ -20,6 +20,25 @@ namespace gnnpre {
 
 namespace {
 
+// The optional teleport term: a finished row r_i * sum becomes keep * (r_i * sum) + alpha * X_0[i].
+struct Teleport {
+    const float* x0;
+    int64_t ldx0;
+    float alpha, keep;  // keep = 1 - alpha
+};
+
+__device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, const Teleport& tp, int64_t row, int q) {
+    float4 o = make_float4(sum.x * scale, sum.y * scale, sum.z * scale, sum.w * scale);
+    if (tp.alpha != 0.f) {
+        const float4 z = __ldg(reinterpret_cast<const float4*>(tp.x0 + row * tp.ldx0) + q);
+        o.x = fmaf(tp.keep, o.x, tp.alpha * z.x);
+        o.y = fmaf(tp.keep, o.y, tp.alpha * z.y);
+        o.z = fmaf(tp.keep, o.z, tp.alpha * z.z);
+        o.w = fmaf(tp.keep, o.w, tp.alpha * z.w);
+    }
+    return o;
+}
+
 struct SegArgs {
     const Segment* segs;
     int64_t seg_lo, seg_hi;
@@ -36,6 +55,7 @@ struct SegArgs {
     const int32_t* nzrows;
     int32_t f4;  // float4 per row of this column tile
     float diag_weight;  // GIN: 1 + eps
+    Teleport tp;
 };
 
 // Compensated (Kahan) addition of x into the pair (sum, comp): the low-order bits that the addition
@@ -160,24 +180,15 @@ __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(co
                     // last edge of a row (never set on a padding lane): the whole group arrives here together
                     const int row = __shfl_sync(gmask, my_row, gshift + t);
                     const float r = __shfl_sync(gmask, my_r, gshift + t);
-                    float* dst;
-                    float scale;
-                    if (head_pending) {  // the row began earlier: leave the partial sum for the fix-up
-                        dst = a.scratch + (int64_t)slot_head * a.scratch_ld;
-                        scale = 1.f;
-                        head_pending = false;
-                    } else {
-                        dst = a.out + (int64_t)row * a.ldo;
-                        scale = r;
-                    }
+                    const bool partial = head_pending;  // the row began earlier: leave the sum for the fix-up
+                    head_pending = false;
+                    float* dst = partial ? a.scratch + (int64_t)slot_head * a.scratch_ld : a.out + (int64_t)row * a.ldo;
 #pragma unroll
                     for (int v = 0; v < V; ++v) {
                         kahan4(tot[v], cmp[v], acc[v]);
-                        if (on[v]) {
-                            float4 o = tot[v];
-                            o.x *= scale; o.y *= scale; o.z *= scale; o.w *= scale;
-                            reinterpret_cast<float4*>(dst)[gl + v * G] = o;
-                        }
+                        if (on[v])
+                            reinterpret_cast<float4*>(dst)[gl + v * G] =
+                                partial ? tot[v] : finish_row_piece(tot[v], r, a.tp, row, gl + v * G);
                         acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
@@ -232,6 +243,7 @@ struct FixArgs {
     float* out;
     int64_t ldo;
     int32_t f4;
+    Teleport tp;
 };
 
 // One group per cut row: tail part of its first segment, then the head parts of the following ones,
@@ -282,22 +294,20 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int q = gl + v * G;
-            if (q < a.f4) {
-                float4 o = acc[v];
-                o.x *= r; o.y *= r; o.z *= r; o.w *= r;
-                *reinterpret_cast<float4*>(dst + 4 * q) = o;
-            }
+            if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = finish_row_piece(acc[v], r, a.tp, row, q);
         }
     }
 }
 
 // Rows without any edge (SAGE, D_i = 0) are zero rows of the result.
+// (With a teleport term they keep alpha * X_0[i].)
 __global__ void k_zero_rows(const int32_t* __restrict__ rows, int64_t count, float* __restrict__ out, int64_t ldo,
-                            int32_t f4) {
+                            int32_t f4, const Teleport tp) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count * f4) return;
     const int64_t r = rows[t / f4];
-    *reinterpret_cast<float4*>(out + r * ldo + 4 * (t % f4)) = make_float4(0.f, 0.f, 0.f, 0.f);
+    const int q = (int)(t % f4);
+    *reinterpret_cast<float4*>(out + r * ldo + 4 * q) = finish_row_piece(make_float4(0.f, 0.f, 0.f, 0.f), 0.f, tp, r, q);
 }
 
 template <int G, int V, int U>
@@ -404,6 +414,15 @@ int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
 
 constexpr int kMaxTile = 512;  // columns one launch covers (G = 32, V = 4)
 
+Teleport teleport_of(const gnnpre_plan* P, const HopArgs& h, int32_t f0) {
+    Teleport tp;
+    tp.x0 = h.x0 ? h.x0 + f0 : nullptr;
+    tp.ldx0 = h.ldx0;
+    tp.alpha = h.x0 ? P->teleport_alpha : 0.f;
+    tp.keep = (float)(1.0 - (double)tp.alpha);
+    return tp;
+}
+
 }  // namespace
 
 // Rows of 68..128 columns (17..32 float4) go through the bulk-copy kernel unless the plan says otherwise.
@@ -433,6 +452,7 @@ int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int6
         a.nzrows = P->nzrows.p;
         a.f4 = w / 4;
         a.diag_weight = 1.0f + P->gin_eps;
+        a.tp = teleport_of(P, h, f0);
         if (uses_bulk_copy(P, w)) GNNPRE_TRY(launch_segments_tma(P, a, st));
         else if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
         else if (a.f4 <= 8) GNNPRE_TRY((launch_segments_shape<8, 1, 8>(P, a, st)));
@@ -459,6 +479,7 @@ int launch_fixups(const gnnpre_plan* P, const HopArgs& h, int64_t fix_lo, int64_
         a.out = h.xout + f0;
         a.ldo = h.ldo;
         a.f4 = w / 4;
+        a.tp = teleport_of(P, h, f0);
         if (a.f4 <= 4) GNNPRE_TRY((launch_fixups_shape<4, 1>(a, st)));
         else if (a.f4 <= 8) GNNPRE_TRY((launch_fixups_shape<8, 1>(a, st)));
         else if (a.f4 <= 16) GNNPRE_TRY((launch_fixups_shape<16, 1>(a, st)));
@@ -473,7 +494,8 @@ int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t 
     if (P->num_empty == 0) return GNNPRE_OK;
     const int32_t f4 = h.width / 4;
     const int64_t items = P->num_empty * f4;
-    k_zero_rows<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4);
+    k_zero_rows<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4,
+                                                                    teleport_of(P, h, 0));
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }
@@ -502,6 +524,8 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
             h.colx = P->colx.p;
             h.colx_edge_base = 0;
             h.xprev = xprev + f_lo;
+            h.x0 = X + f_lo;
+            h.ldx0 = ldx;
             h.ldx = ldp;
             h.xout = out[k] + f_lo;
             h.ldo = ldo;

@@ -228,20 +228,14 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
         auto flush = [&](int t, const TmaChunk& m) {
             const int row = __shfl_sync(kFull, m.row, t);
             const float r = __shfl_sync(kFull, m.r, t);
-            float* dst;
-            float scale;
-            if (head_pending) {
-                dst = a.scratch + (int64_t)slot_head * a.scratch_ld;
-                scale = 1.f;
-                head_pending = false;
-            } else {
-                dst = a.out + (int64_t)row * a.ldo;
-                scale = r;
-            }
+            const bool partial = head_pending;  // the row began in an earlier segment: leave the sum for the fix-up
+            head_pending = false;
+            float* dst = partial ? a.scratch + (int64_t)slot_head * a.scratch_ld : a.out + (int64_t)row * a.ldo;
             quad_kahan(tot, cmp, acc);
-            if (on)
-                reinterpret_cast<float4*>(dst)[lane] =
-                    make_float4(tot.lo.x * scale, tot.lo.y * scale, tot.hi.x * scale, tot.hi.y * scale);
+            if (on) {
+                const float4 sum = make_float4(tot.lo.x, tot.lo.y, tot.hi.x, tot.hi.y);
+                reinterpret_cast<float4*>(dst)[lane] = partial ? sum : finish_row_piece(sum, r, a.tp, row, lane);
+            }
             acc = tot = cmp = quad_zero();
         };
 

@@ -118,6 +118,8 @@ int run(gnnpre_plan* P, const float* X, int64_t ldx, bool x_host, int32_t K, flo
             }
             HopArgs h;
             h.xprev = xprev;
+            h.x0 = x_host ? in[i & 1].p : X + f_lo;  // the slab of X_0 stays put for all K hops
+            h.ldx0 = x_host ? w : ldx;
             h.ldx = ldp;
             h.xout = xout;
             h.ldo = ldd;
@@ -158,6 +160,7 @@ int run(gnnpre_plan* P, const float* X, int64_t ldx, bool x_host, int32_t K, flo
                     d2h += 4 * width * rows;
                 }
                 if (j + 1 == P->blocks.size()) {
+                    if (x_host) in[i & 1].kernel_read = done;  // every hop may read X_0's slab (teleport term)
                     if (prev_buf) prev_buf->kernel_read = done;
                     if (dst_buf) {
                         dst_buf->filled = done;

@@ -381,3 +381,36 @@ def test_a_device_wait_that_runs_out_is_reported_and_leaves_the_plan_usable(B):
     outs, st = B.gnnpre_propagate(plan, X, 2, want_stats=True)  # the error word was cleared: no stale timeout
     check_all_hops(0, 0.0, rp, ci, to_np(X), outs)
     plan.close()
+
+
+# ------------------------------------------------------------------ teleport (personalised PageRank) filter
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("alpha", [0.15, 1.0])
+def test_teleport_filter_matches_oracle(B, op, alpha):
+    """X_k = (1 - alpha) A^ X_{k-1} + alpha X_0 for every kernel shape, with blocks and slabs, resident and
+    streamed (bitwise equal to each other), against the fp64 oracle."""
+    g = gi.rmat(6000, 60000, 27, directed_candidates=True)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    K = 3
+    for F, b, c in ((16, 1, 1), (100, 3, 1), (128, 2, 2), (256, 1, 1), (72, 4, 3)):
+        X = gi.normal_matrix(g.n, F, 7, device="cuda")
+        want = orc.propagate_teleport(op, EPS, alpha, rp, ci, to_np(X), K)
+        plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c, segment_edges=64,
+                                   teleport_alpha=alpha)
+        outs, _ = B.gnnpre_propagate(plan, X, K)
+        torch.cuda.synchronize()
+        for k in range(K):
+            assert hop_error(to_np(outs[k]), want[k]) <= TOL, (F, b, c, k)
+        hplan = B.gnnpre_build_plan(g.rowptr.pin_memory(), g.colidx.pin_memory(), op, F, gin_eps=EPS, force_blocks=b,
+                                    force_col_slabs=c, segment_edges=64, teleport_alpha=alpha,
+                                    operands_mem=B.GNNPRE_MEM_HOST)
+        houts = [torch.empty(g.n, F).pin_memory() for _ in range(K)]
+        B.gnnpre_propagate(hplan, X.cpu().pin_memory(), K, houts)
+        for k in range(K):
+            assert torch.equal(houts[k], outs[k].cpu()), (F, b, c, k)
+        plan.close()
+        hplan.close()
+    with pytest.raises(B.GnnpreError):
+        B.gnnpre_build_plan(drp, dci, op, 16, teleport_alpha=1.5)
