@@ -1,12 +1,12 @@
 // Segment kernel with the gathered rows staged through shared memory by the bulk-copy (TMA) engine.
 // Included by propagate.cu inside its unnamed namespace (uses SegArgs, Segment, kRowEndBit).
 //
-// Why: the register kernel k_segments keeps at most (warps per SM) x U rows in flight, bounded by
-// the register file; a gather of 400-512 B rows at random addresses needs ~100 KB in flight per SM
-// to hide HBM/L2 latency.  Here every lane of a warp asks the copy engine for one neighbour row
-// (cp.async.bulk, global -> shared, completion counted in bytes on an mbarrier), so a warp has up
-// to kTmaStages x 32 rows in flight and they occupy shared memory (up to ~220 KB per SM) instead of
-// registers.  The warp then sums the rows out of shared memory with conflict-free 128-bit reads.
+// Why: the register kernel k_segments keeps at most (warps per SM) x 8 rows in flight, bounded by
+// the register file and the load/store path; a gather of 400-512 B rows at random addresses needs on
+// the order of 100 KB in flight per SM to hide HBM/L2 latency.  Here the copy engine moves the rows
+// (completion counted in bytes on an mbarrier) and they wait in shared memory - kTmaStages x kTmaRows
+// rows per warp, about 210 KB per SM - instead of registers.  The warp then sums the rows out of
+// shared memory with conflict-free 128-bit reads.
 //
 // One CTA per SM, persistent: warp w of the grid walks segments w, w + W, w + 2W, ... (W = warps in
 // the grid), so no atomics are involved and the summation order is the same as in k_segments
