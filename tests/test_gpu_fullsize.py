@@ -77,6 +77,10 @@ def test_config5_scaled_streamed_with_budget(B):
     _, st = B.gnnpre_propagate(plan, Xh, K, outs, want_stats=True)
     assert st.d2h_bytes == 4 * g.n * F * K
     assert st.h2d_bytes >= 4 * g.n * F + 4 * m  # X once, and E at least once
+    # Eq. 12 is a model: what the plan really holds on the device after a streamed call (edge-block staging
+    # buffers, four slab buffers, per-node arrays, row pointers, segment tables) stays within 10 % of the budget
+    used = plan.info()["device_bytes"]
+    assert used <= 1.10 * budget, (used, budget)
     ref_plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, force_blocks=info["b"], force_col_slabs=info["c"],
                                    segment_edges=info["segment_edges"])
     ref, _ = B.gnnpre_propagate(ref_plan, X, K)
