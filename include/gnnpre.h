@@ -143,6 +143,8 @@ int gnnpre_degrees(const gnnpre_csr_t* csr, int32_t* deg_out, void* stream);
  * with self-loops inserted at their sorted position, (b, c) from Eq. 12 unless forced, the b
  * balanced contiguous edge blocks  [floor(l|E|/b), floor((l+1)|E|/b))  and the warp-level segment
  * tables.  Synchronous.  The plan is immutable afterwards; free it with gnnpre_plan_destroy.
+ * While it runs, the build holds the CSR and some flag arrays on the device besides the plan itself
+ * (a host-resident CSR is copied there for the duration): about 2 * B_S transient bytes.
  * Errors: INVALID_ARG (NULLs, bad op, F < 4, b > |E|, c > ceil(F/4)), ALIGN (F % 4 != 0),
  * INVALID_CSR, BUDGET_TOO_SMALL, OOM_*, CUDA, UNSUPPORTED_ARCH.
  */
@@ -178,6 +180,9 @@ int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t*
  * Accumulation is fp32 in a fixed order: results are bitwise reproducible from run to run for a
  * given plan, and agree across different (b, c) or segment sizes only to rounding.
  * `stats` may be NULL; when given, device-resident calls synchronise `stream` to read the timers.
+ * Resuming: every hop depends on the previous one only, so a run interrupted after hop k continues by
+ * calling again with X = out[k-1] and K' = K - k (plain filters; bit-identical to the uninterrupted run).
+ * With a teleport term X must be X_0, so a resumed run starts from hop 1.
  */
 int gnnpre_propagate(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t x_mem, int32_t K, float* const* out,
                      int64_t ldo, int32_t out_mem, void* stream, gnnpre_stats_t* stats);

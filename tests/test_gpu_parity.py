@@ -414,3 +414,16 @@ def test_teleport_filter_matches_oracle(B, op, alpha):
         hplan.close()
     with pytest.raises(B.GnnpreError):
         B.gnnpre_build_plan(drp, dci, op, 16, teleport_alpha=1.5)
+
+
+def test_resuming_from_a_finished_hop_gives_the_same_bits(B):
+    """Checkpoint/resume: hops 1..2, then hop 3 started from hop 2's output, equal the uninterrupted run."""
+    g = gi.rmat(20000, 200000, 29, directed_candidates=True)
+    plan = B.gnnpre_build_plan(*dev(g), 1, 100, force_blocks=3)
+    X = gi.normal_matrix(g.n, 100, 4, device="cuda")
+    full, _ = B.gnnpre_propagate(plan, X, 3)
+    first, _ = B.gnnpre_propagate(plan, X, 2)
+    rest, _ = B.gnnpre_propagate(plan, first[1], 1)
+    torch.cuda.synchronize()
+    assert torch.equal(first[0], full[0]) and torch.equal(first[1], full[1]) and torch.equal(rest[0], full[2])
+    plan.close()
