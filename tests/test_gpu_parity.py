@@ -133,7 +133,7 @@ def test_config1_erdos_renyi_gcn(B):
 @pytest.mark.parametrize("op", OPS)
 def test_small_graphs_all_shapes(B, name, g, op):
     m = orc.support_nnz(op, g.n, g.nnz)
-    for F, seg in ((4, 8), (16, 4), (20, 32), (64, 8), (100, 16), (128, 0), (256, 8), (516, 32), (1040, 8)):
+    for F, seg in ((4, 8), (16, 4), (20, 32), (64, 8), (100, 16), (128, 0), (256, 8), (516, 32), (640, 16), (1040, 8)):
         for b in (1, 3):
             if b > m:
                 continue
@@ -427,3 +427,19 @@ def test_resuming_from_a_finished_hop_gives_the_same_bits(B):
     torch.cuda.synchronize()
     assert torch.equal(first[0], full[0]) and torch.equal(first[1], full[1]) and torch.equal(rest[0], full[2])
     plan.close()
+
+
+@pytest.mark.parametrize("op", OPS)
+def test_streamed_slabs_through_the_bulk_copy_kernel(B, op):
+    """Column slabs of 100 columns (F = 200, c = 2) and a 128-column tail tile (F = 640): the tensor map of the
+    bulk-copy kernel starts at a column offset, in dense slab buffers and in the caller's strided matrix."""
+    g = gi.rmat(12000, 150000, 31, directed_candidates=True)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    for F, c in ((200, 2), (640, 1)):
+        X = gi.normal_matrix(g.n, F, 8, device="cuda")
+        plan = B.gnnpre_build_plan(*dev(g), op, F, gin_eps=EPS, force_blocks=3, force_col_slabs=c,
+                                   operands_mem=B.GNNPRE_MEM_HOST)
+        houts = [torch.empty(g.n, F).pin_memory() for _ in range(2)]
+        B.gnnpre_propagate(plan, X.cpu().pin_memory(), 2, houts)
+        check_all_hops(op, EPS, rp, ci, to_np(X), houts)
+        plan.close()
