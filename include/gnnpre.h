@@ -35,7 +35,7 @@ typedef enum {
     GNNPRE_OK = 0,
     GNNPRE_ERR_INVALID_ARG = -1,      /* NULL pointer, bad enum, bad size, b > |E| ... */
     GNNPRE_ERR_INVALID_CSR = -2,      /* see gnnpre_csr_t */
-    GNNPRE_ERR_ALIGN = -3,            /* pointer not 16-byte aligned, or a leading dimension / F not a multiple of 4 */
+    GNNPRE_ERR_ALIGN = -3,            /* pointer not 16-byte aligned, or a leading dimension not a multiple of 4 */
     GNNPRE_ERR_OOM_DEVICE = -4,
     GNNPRE_ERR_OOM_HOST = -5,
     GNNPRE_ERR_BUDGET_TOO_SMALL = -6, /* Eq. 12 has no feasible (b, c) */
@@ -74,7 +74,9 @@ typedef struct {
 typedef struct {
     int32_t op;              /* gnnpre_op_t */
     float gin_eps;           /* GIN_SUM only */
-    int64_t feat_dim;        /* F: columns of X; must be a multiple of 4 */
+    int64_t feat_dim;        /* F: columns of X.  Work is done on whole groups of 4 columns: with F % 4 != 0 the
+                                1..3 pad columns up to the next multiple of 4 (which ldx, ldo >= that multiple
+                                make room for) are read from X and written to out[] with unspecified values */
     int64_t budget_bytes;    /* B_GPU of Eq. 12; 0 = the device's free memory at plan time */
     int32_t force_blocks;    /* b; 0 = solve Eq. 12 */
     int32_t force_col_slabs; /* c; 0 = solve Eq. 12 */
@@ -93,7 +95,7 @@ typedef struct gnnpre_plan gnnpre_plan_t; /* opaque; owns device (and pinned hos
 
 typedef struct {
     int64_t n, nnz, nnz_tilde; /* nnz_tilde = |E|: nnz + n for GCN/GIN (self-loops are edges of E), nnz for SAGE */
-    int64_t feat_dim;
+    int64_t feat_dim;          /* F rounded up to a multiple of 4 */
     int32_t op;
     int32_t b, c;              /* Eq. 12's block counts in use */
     int64_t slab_width;        /* columns per slab: 4 * ceil(F / (4c)) */
@@ -145,8 +147,7 @@ int gnnpre_degrees(const gnnpre_csr_t* csr, int32_t* deg_out, void* stream);
  * tables.  Synchronous.  The plan is immutable afterwards; free it with gnnpre_plan_destroy.
  * While it runs, the build holds the CSR and some flag arrays on the device besides the plan itself
  * (a host-resident CSR is copied there for the duration): about 2 * B_S transient bytes.
- * Errors: INVALID_ARG (NULLs, bad op, F < 4, b > |E|, c > ceil(F/4)), ALIGN (F % 4 != 0),
- * INVALID_CSR, BUDGET_TOO_SMALL, OOM_*, CUDA, UNSUPPORTED_ARCH.
+ * Errors: INVALID_ARG (NULLs, bad op, F < 1, b > |E|, c > ceil(F/4)), INVALID_CSR, BUDGET_TOO_SMALL, OOM_*, CUDA, UNSUPPORTED_ARCH.
  */
 int gnnpre_build_plan(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpre_plan_opts_t* opts,
                       gnnpre_plan_t** plan_out);
@@ -168,7 +169,8 @@ int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t*
  * teleport term in the plan, out[k-1] <- (1 - alpha) A^ out[k-2] + alpha X instead.
  *   X      fp32 row-major [n, F] with leading dimension ldx (floats), in x_mem
  *   out    host array of K pointers, each fp32 row-major [n, F] with leading dimension ldo, in out_mem
- *   ldx, ldo >= F and multiples of 4; all base pointers 16-byte aligned (else GNNPRE_ERR_ALIGN)
+ *   ldx, ldo >= F rounded up to a multiple of 4 (else INVALID_ARG), themselves multiples of 4, and all base
+ *   pointers 16-byte aligned (else GNNPRE_ERR_ALIGN)
  *   out[k] must not overlap X or another out[]; 1 <= K <= GNNPRE_MAX_HOPS
  * Device X and device out: the work is enqueued on `stream` and the call returns at once; the
  * plan's scratch memory is in use until that work completes, so calls on one plan must not

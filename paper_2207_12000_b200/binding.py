@@ -206,10 +206,11 @@ def gnnpre_propagate(plan: Plan, X: torch.Tensor, K: int, out: Sequence[torch.Te
     assert X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
     n, F = X.shape
     if out is None:
+        Fp = (F + 3) // 4 * 4  # the library works on whole groups of 4 columns
         if X.is_cuda:
-            out = [torch.empty((n, F), dtype=torch.float32, device=X.device) for _ in range(K)]
+            out = [torch.empty((n, Fp), dtype=torch.float32, device=X.device)[:, :F] for _ in range(K)]
         else:
-            out = [torch.empty((n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
+            out = [torch.empty((n, Fp), dtype=torch.float32, pin_memory=True)[:, :F] for _ in range(K)]
     assert len(out) == K
     ldo = out[0].stride(0) if K > 0 else F
     for o in out:

@@ -437,7 +437,7 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     P->n = n;
     P->nnz = nnz;
     P->nnz_tilde = nnz + (diag ? n : 0);
-    P->feat_dim = opts->feat_dim;
+    P->feat_dim = (opts->feat_dim + 3) / 4 * 4;  // whole float4 columns; the caller's leading dimensions cover the pad
     P->op = opts->op;
     P->gin_eps = opts->gin_eps;
     P->teleport_alpha = opts->teleport_alpha;
@@ -746,8 +746,7 @@ extern "C" int gnnpre_build_plan(const gnnpre_csr_t* csr, const int32_t* degrees
     if (opts->op < GNNPRE_OP_GCN_SYM || opts->op > GNNPRE_OP_GIN_SUM) return GNNPRE_ERR_INVALID_ARG;
     if (opts->operands_mem != GNNPRE_MEM_DEVICE && opts->operands_mem != GNNPRE_MEM_HOST) return GNNPRE_ERR_INVALID_ARG;
     if (!(opts->teleport_alpha >= 0.f && opts->teleport_alpha <= 1.f)) return GNNPRE_ERR_INVALID_ARG;
-    if (opts->feat_dim < 4) return GNNPRE_ERR_INVALID_ARG;
-    if (opts->feat_dim % 4 != 0) return GNNPRE_ERR_ALIGN;
+    if (opts->feat_dim < 1) return GNNPRE_ERR_INVALID_ARG;
     if (opts->segment_edges < 0 || opts->segment_edges > (1 << 20)) return GNNPRE_ERR_INVALID_ARG;
     GNNPRE_TRY(check_device());
     gnnpre_plan* P = new (std::nothrow) gnnpre_plan();

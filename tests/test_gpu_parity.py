@@ -223,7 +223,7 @@ def test_invalid_inputs_are_rejected(B):
             fn()
         return ei.value.status
 
-    assert status(lambda: B.gnnpre_build_plan(drp, dci, 0, 18)) == -3          # F % 4
+    assert status(lambda: B.gnnpre_build_plan(drp, dci, 0, 0)) == -1           # F < 1
     assert status(lambda: B.gnnpre_build_plan(drp, dci, 5, 16)) == -1          # bad op
     assert status(lambda: B.gnnpre_build_plan(drp, dci, 1, 16, force_blocks=g.nnz + 1)) == -1  # empty block
     assert status(lambda: B.gnnpre_build_plan(drp, dci, 0, 16, force_col_slabs=5)) == -1
@@ -443,3 +443,22 @@ def test_streamed_slabs_through_the_bulk_copy_kernel(B, op):
         B.gnnpre_propagate(plan, X.cpu().pin_memory(), 2, houts)
         check_all_hops(op, EPS, rp, ci, to_np(X), houts)
         plan.close()
+
+
+def test_feature_width_that_is_not_a_multiple_of_four(B):
+    """F = 602 (Reddit's width in the paper's dataset table): the matrices carry a leading dimension of 604; the
+    two pad columns may hold anything (NaN here) without touching the 602 real ones."""
+    g = gi.erdos_renyi(3000, 30000, 33)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    F, ld = 602, 604
+    Xbuf = torch.full((g.n, ld), float("nan"), device="cuda")
+    Xbuf[:, :F] = gi.normal_matrix(g.n, F, 3, device="cuda")
+    obuf = [torch.zeros((g.n, ld), device="cuda") for _ in range(2)]
+    plan = B.gnnpre_build_plan(*dev(g), 0, F, force_blocks=2)
+    assert plan.info()["feat_dim"] == 604
+    B.gnnpre_propagate(plan, Xbuf[:, :F], 2, [o[:, :F] for o in obuf])
+    torch.cuda.synchronize()
+    check_all_hops(0, 0.0, rp, ci, to_np(Xbuf[:, :F]).copy(), [o[:, :F] for o in obuf])
+    with pytest.raises(B.GnnpreError):  # no room for the pad columns
+        B.gnnpre_propagate(plan, torch.zeros((g.n, F), device="cuda")[:, :F], 1)
+    plan.close()
