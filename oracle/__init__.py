@@ -63,6 +63,7 @@ def _c():
         lib.orc_slab_width.restype = i64
         lib.orc_propagate_blocked.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, ctypes.c_int, i32, i32, p]
         lib.orc_propagate_blocked.restype = ctypes.c_int
+        lib.orc_lc_first_layer.argtypes = [i64, p, i64, p, i64, i64, p, i64, ctypes.c_int, p, p]
         _lib = lib
     return _lib
 
@@ -217,3 +218,22 @@ def propagate_blocked(op: int, eps: float, rowptr, colidx, X, K: int, b: int, c:
     if rc != 0:
         raise ValueError("impossible (b, c)")
     return out
+
+
+def lc_first_layer(Xk, batch, Wt, relu: bool, want_abs: bool = False):
+    """act(Xk[batch] @ Wt.T) in fp64 (Eq. 9's first dense stage); Wt is [H, F]; batch None = all rows."""
+    Xk, ldx = _f32_matrix(Xk)
+    Wt, ldw = _f32_matrix(Wt)
+    F, H = Xk.shape[1], Wt.shape[0]
+    assert Wt.shape[1] == F
+    if batch is None:
+        B, bp = Xk.shape[0], None
+    else:
+        batch = np.ascontiguousarray(batch, dtype=np.int64)
+        assert batch.size == 0 or (batch.min() >= 0 and batch.max() < Xk.shape[0])
+        B, bp = batch.shape[0], _ptr(batch)
+    Y = np.empty((B, H), dtype=np.float64)
+    A = np.empty((B, H), dtype=np.float64) if want_abs else None
+    _c().orc_lc_first_layer(B, bp, F, _ptr(Xk), ldx, H, _ptr(Wt), ldw, int(bool(relu)), _ptr(Y),
+                            _ptr(A) if want_abs else None)
+    return (Y, A) if want_abs else Y

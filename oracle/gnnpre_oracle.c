@@ -25,6 +25,8 @@
  * Parity pins (tests/test_oracle_pins.py): closed forms on complete, cycle, star and regular
  * graphs, fixed points and conservation laws of each operator, brute-force dense A^^k X,
  * an independent scipy.sparse product, and exhaustive checks of the block partition.
+ * The first dense stage of an LC model (Eq. 9), orc_lc_first_layer, is pinned by a library matrix
+ * product, by one-hot / identity weights and by the commutation S^k (X W) = (S^k X) W on integers.
  * Absolute speed is the one thing with no pin: the paper prints ratios only.
  */
 #include <math.h>
@@ -406,4 +408,35 @@ int orc_propagate_blocked(int op, double eps, int64_t n, const int64_t* rowptr, 
     free(deg);
     free(e_off);
     return 0;
+}
+
+/* ------------------------------------------------------------------ first dense stage of an LC model */
+
+/*
+ * Eq. 9 (the LC version of JKNet): every term of COMB starts with  S^k X W_1 , the k-th
+ * precomputed hop times the first weight matrix, followed by the activation sigma (ReLU in
+ * the paper's experimental settings) whenever another layer follows.  Training runs on
+ * mini-batches of rows (batch size 4096 in the settings), so the stage is
+ *     Y[i][h] = act( sum_f  Xk[batch[i]][f] * Wt[h][f] ),   i < B, h < H,
+ * with Wt the weight stored as [H, F] (one row per output unit).  `batch` == NULL means rows
+ * 0..B-1.  Yabs, when given, receives sum_f |Xk| |Wt| (the scale of the rounding error of any
+ * finite-precision evaluation).  fp64 throughout, f ascending.
+ */
+void orc_lc_first_layer(int64_t B, const int64_t* batch, int64_t F, const float* Xk, int64_t ldx, int64_t H,
+                        const float* Wt, int64_t ldw, int relu, double* Y, double* Yabs) {
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < B; ++i) {
+        const float* x = Xk + (batch ? batch[i] : i) * ldx;
+        for (int64_t h = 0; h < H; ++h) {
+            const float* w = Wt + h * ldw;
+            double s = 0.0, a = 0.0;
+            for (int64_t f = 0; f < F; ++f) {
+                s += (double)x[f] * (double)w[f];
+                a += fabs((double)x[f]) * fabs((double)w[f]);
+            }
+            if (relu && s < 0.0) s = 0.0;
+            Y[i * H + h] = s;
+            if (Yabs) Yabs[i * H + h] = a;
+        }
+    }
 }

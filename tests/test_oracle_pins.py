@@ -497,3 +497,48 @@ def test_teleport_on_complete_graph_closed_form():
     got = orc.propagate_teleport(orc.OP_GCN, 0.0, a, rowptr, colidx, X, 4)
     for k in range(4):
         np.testing.assert_allclose(got[k], want, rtol=1e-13, atol=1e-15)
+
+
+# ------------------------------------------------------------------ first dense stage of an LC model (Eq. 9)
+
+def test_first_layer_against_library_product_and_special_weights():
+    n, F, H = 90, 13, 7  # H != F so that a transposed weight cannot pass
+    X, Wt = features(n, F, 61), features(H, F, 62)
+    batch = np.random.default_rng(5).integers(0, n, size=41)
+    Y, A = orc.lc_first_layer(X, batch, Wt, relu=False, want_abs=True)
+    ref = X[batch].astype(np.float64) @ Wt.astype(np.float64).T
+    np.testing.assert_allclose(Y, ref, rtol=1e-13, atol=1e-14)
+    np.testing.assert_allclose(A, np.abs(X[batch]).astype(np.float64) @ np.abs(Wt).astype(np.float64).T, rtol=1e-13)
+    assert (np.abs(Y) <= A * (1 + 1e-12)).all()
+    # sigma = ReLU applied after the product, element by element
+    R = orc.lc_first_layer(X, batch, Wt, relu=True)
+    np.testing.assert_array_equal(R, np.maximum(Y, 0.0))
+    assert (R == 0).any() and (R > 0).any()
+    # one-hot weights pick columns; the identity returns the gathered rows; no batch = every row in order
+    sel = np.zeros((3, F), dtype=np.float32)
+    sel[0, 4] = sel[1, 0] = sel[2, 12] = 1.0
+    np.testing.assert_array_equal(orc.lc_first_layer(X, batch, sel, relu=False), X[batch][:, [4, 0, 12]].astype(np.float64))
+    np.testing.assert_array_equal(orc.lc_first_layer(X, None, np.eye(F, dtype=np.float32), relu=False), X.astype(np.float64))
+    # a strided matrix (leading dimension above F) is honoured
+    Xs = np.full((n, F + 3), np.nan, dtype=np.float32)
+    Xs[:, :F] = X
+    np.testing.assert_array_equal(orc.lc_first_layer(Xs[:, :F], batch, Wt, relu=False), Y)
+    assert orc.lc_first_layer(X, np.zeros(0, dtype=np.int64), Wt, relu=True).shape == (0, H)
+
+
+def test_first_layer_commutes_with_propagation():
+    """The LC transformation rests on S^k (X W) = (S^k X) W.  With the GIN sum operator (eps = 0) and
+    small integer X, W every quantity is an integer that fp32 holds exactly, so both sides are equal."""
+    n, F, H, K = 60, 6, 4, 3
+    rowptr, colidx = random_graph(n, 150, 71)
+    rng = np.random.default_rng(72)
+    X = rng.integers(-3, 4, size=(n, F)).astype(np.float32)
+    Wt = rng.integers(-2, 3, size=(H, F)).astype(np.float32)
+    hops = orc.propagate(orc.OP_GIN, 0.0, rowptr, colidx, X, K)
+    XW = (X.astype(np.float64) @ Wt.astype(np.float64).T).astype(np.float32)
+    hops_of_XW = orc.propagate(orc.OP_GIN, 0.0, rowptr, colidx, XW, K)
+    batch = rng.permutation(n)[:37]
+    for k in range(K):
+        hop32 = hops[k].astype(np.float32)
+        assert (hop32.astype(np.float64) == hops[k]).all()
+        np.testing.assert_array_equal(orc.lc_first_layer(hop32, batch, Wt, relu=False), hops_of_XW[k][batch])
