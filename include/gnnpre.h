@@ -251,6 +251,40 @@ void gnnpre_plan_destroy(gnnpre_plan_t* plan);
 int gnnpre_hop_static(const gnnpre_csr_t* csr, int32_t op, float gin_eps, int64_t feat_dim, const float* X,
                       int64_t ldx, float* out, int64_t ldo, void* stream);
 
+/*
+ * First dense stage of an LC model on a mini-batch of rows (Eq. 9: every term of COMB begins with the
+ * k-th precomputed hop times the first weight matrix; the experimental settings use mini-batches of
+ * 4096 rows, hidden width 256 and ReLU).  For each hop matrix k < num_hops:
+ *
+ *     Y_k[i][h] = act_k( sum_f hops[k][batch[i]][f] * Wt[h][f] ),   i < batch_size, h < hidden,
+ *
+ * act_k = ReLU if bit k of relu_mask is set, else the identity.  The batch rows are gathered by the
+ * operand loads of the matrix product; no [batch_size, feat_dim] copy is made.
+ *
+ *   hops       HOST array of num_hops DEVICE pointers, each fp32 row-major [n, feat_dim] with leading
+ *              dimension ldh (the out[] of gnnpre_propagate, or X_0); 1 <= num_hops <= GNNPRE_MAX_HOPS
+ *   batch      DEVICE int32[batch_size], row of the hop matrices per output row; NULL = rows
+ *              0..batch_size-1 (then batch_size <= n).  NOT validated: an index outside [0, n) reads
+ *              as a row of zeros
+ *   Wt         DEVICE fp32 [hidden, feat_dim], leading dimension ldw: one row per output unit (the
+ *              transpose of Eq. 9's W_1); hidden a multiple of 16, 16 <= hidden <= 256
+ *   Y          DEVICE fp32; element (k, i, h) at Y[k * y_hop_stride + i * ldy + h].  y_hop_stride =
+ *              batch_size * ldy stacks the hops; y_hop_stride = hidden with ldy = num_hops * hidden
+ *              lays them side by side in one row (COMB = concatenation)
+ *   error_flag DEVICE int32 or NULL; set to 1 by the kernel if one of its bounded waits ran out
+ *              (the results are then invalid).  The caller clears and reads it.
+ * ldh, ldw >= feat_dim and ldy >= hidden (else INVALID_ARG); ldh, ldw, ldy, y_hop_stride multiples of 4
+ * and all base pointers 16-byte aligned (else ALIGN).  feat_dim itself may be any value >= 1.
+ * Arithmetic: tensor cores with tf32 inputs (the fp32 operands are read with their low 13 mantissa
+ * bits ignored) and fp32 accumulation: |error| <= 2^-9 * sum_f |x||w| plus fp32 summation error.
+ * The work is enqueued on `stream` and the call returns without synchronising; nothing is allocated.
+ * batch_size = 0 is a no-op.  UNSUPPORTED_ARCH on devices other than compute capability 10.x.
+ */
+int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
+                          const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw,
+                          uint64_t relu_mask, float* Y, int64_t ldy, int64_t y_hop_stride, int32_t* error_flag,
+                          void* stream);
+
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;
  * ties towards smaller c, then smaller b.  BUDGET_TOO_SMALL if infeasible.  Host only. */

@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
                                      ctypes.POINTER(gnnpre_stats_t)]
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
+    lib.gnnpre_lc_first_layer.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i64, i64, i64, p, i64, p, i64, i64,
+                                          ctypes.c_uint64, p, i64, i64, p, p]
     lib.gnnpre_normalize.argtypes = [p, p, i32, p]
     lib.gnnpre_solve_normalisation_blocks.argtypes = [i64] * 8 + [ctypes.POINTER(i64)]
     lib.gnnpre_selftest_wait_timeout.argtypes = [p, ctypes.c_uint32, p]
@@ -236,6 +238,43 @@ def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: to
     return out
 
 
+def gnnpre_lc_first_layer(hops, batch, Wt: torch.Tensor, *, relu_mask: int = 0, out: torch.Tensor | None = None,
+                          concat: bool = False, check: bool = True, stream=None) -> torch.Tensor:
+    """act(hops[k][batch] @ Wt.T) for every hop on the tensor cores (Eq. 9's first dense stage).
+
+    hops: list of device fp32 [n, F] matrices with one common row stride; batch: device int32 row indices
+    or None (all rows); Wt: device fp32 [H, F].  Returns [K, B, H], or [B, K*H] with concat=True.
+    With check=True the call synchronises and raises if a device-side wait ran out."""
+    K = len(hops)
+    n, F = hops[0].shape
+    for h in hops:
+        assert h.is_cuda and h.dtype == torch.float32 and h.shape == (n, F) and h.stride(1) == 1
+        assert h.stride(0) == hops[0].stride(0)
+    assert Wt.is_cuda and Wt.dtype == torch.float32 and Wt.dim() == 2 and Wt.shape[1] == F and Wt.stride(1) == 1
+    H = Wt.shape[0]
+    if batch is None:
+        B, bptr = n, None
+    else:
+        assert batch.is_cuda and batch.dtype == torch.int32 and batch.dim() == 1 and batch.is_contiguous()
+        B, bptr = batch.numel(), batch.data_ptr()
+    if out is None:
+        out = torch.empty((B, K * H) if concat else (K, B, H), dtype=torch.float32, device=Wt.device)
+    if concat:
+        assert out.shape == (B, K * H) and out.stride(1) == 1
+        ldy, hop_stride = out.stride(0), H
+    else:
+        assert out.shape == (K, B, H) and out.stride(2) == 1
+        ldy, hop_stride = (out.stride(1), out.stride(0)) if B > 0 else (H, 0)
+    flag = torch.zeros(1, dtype=torch.int32, device=Wt.device) if check else None
+    ptrs = (ctypes.c_void_p * K)(*[h.data_ptr() for h in hops])
+    _check(_lib.gnnpre_lc_first_layer(ptrs, K, n, F, hops[0].stride(0), bptr, B, Wt.data_ptr(), H, Wt.stride(0),
+                                      relu_mask, out.data_ptr(), ldy, hop_stride,
+                                      flag.data_ptr() if check else None, _stream_ptr(stream)), "gnnpre_lc_first_layer")
+    if check and int(flag.item()) != 0:
+        raise GnnpreError(-8, "gnnpre_lc_first_layer")
+    return out
+
+
 def gnnpre_normalize(plan: Plan, out: torch.Tensor | None = None, *, host: bool = False, stream=None) -> torch.Tensor:
     """fp32 value of every edge of the support (order of gnnpre_plan_support), on the device or in host memory."""
     m = gnnpre_plan_info(plan)["nnz_tilde"]
@@ -277,6 +316,6 @@ def gnnpre_status_string(status: int) -> str:
 
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
-            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_normalize",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_normalize",
             "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

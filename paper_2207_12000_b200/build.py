@@ -6,7 +6,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
-SOURCES = ["plan.cu", "propagate.cu", "stream.cu", "noalloc.cu", "normalize.cu", "api.cu"]
+SOURCES = ["plan.cu", "propagate.cu", "stream.cu", "noalloc.cu", "normalize.cu", "lc_layer.cu", "api.cu"]
 LIB = os.path.join(HERE, "lib", "libgnnpre.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
