@@ -12,9 +12,12 @@
 //            operands read from shared memory through swizzled K-major descriptors, fp32 accumulator
 //            in tensor memory) and hands stages back with tcgen05.commit on the `empty` mbarrier.
 //   warps 2-5  epilogue.  Each warp owns one quarter of the accumulator's 128 lanes, pulls it out of
-//            tensor memory with tcgen05.ld, applies ReLU where asked and stores 64-byte pieces of its
-//            row of Y.
+//            tensor memory with tcgen05.ld 32 columns at a time, applies ReLU where asked, lays the
+//            [32, 32] box down in shared memory (128-byte swizzle, conflict-free) and hands it to the
+//            copy engine as a tensor store, which writes whole lines and clips the ragged edges.
 //
+// A weight of up to 128 KB is loaded once per CTA and stays in shared memory; a larger one is
+// streamed chunk by chunk beside the rows.
 // The accumulator is double-buffered (2 x 256 of the 512 tensor-memory columns), so the epilogue of
 // one tile overlaps the copies and MMAs of the next.  The gathered rows never exist in HBM as a
 // matrix of their own: the gather is the A-operand load.
@@ -37,11 +40,12 @@ namespace {
 
 constexpr int kLcTileM = 128;                     // batch rows per tile = accumulator lanes
 constexpr int kLcChunk = 32;                      // features per stage: 32 fp32 = one 128-byte swizzle row
-constexpr int kLcStages = 4;
+constexpr int kLcMaxStages = 8;
+constexpr int kLcPipeBytes = 192 * 1024;          // operand stages plus, when it fits, the resident weight
+constexpr int kLcResidentMax = 128 * 1024;        // largest weight kept in shared memory for the whole launch
+constexpr int kLcEpiBytes = 32 * 128;             // one [32, 32] fp32 output box
 constexpr int kLcMaxHidden = 256;                 // N of one MMA, columns of one accumulator buffer
 constexpr int kLcABytes = kLcTileM * 128;         // 16 KB
-constexpr int kLcBBytes = kLcMaxHidden * 128;     // 32 KB
-constexpr int kLcStageBytes = kLcABytes + kLcBBytes;
 constexpr int kLcThreads = 192;
 constexpr int kLcMaxHops = 8;                     // hop matrices (tensor maps) per launch
 constexpr uint32_t kLcTmemCols = 512;
@@ -49,8 +53,9 @@ constexpr uint32_t kLcSuspendNs = 20000;          // a failed poll parks the war
 constexpr uint32_t kLcSpinLimit = 50000;          // polls before a wait gives up (about a second)
 
 struct LcMaps {
-    CUtensorMap hop[kLcMaxHops];
-    CUtensorMap w;
+    CUtensorMap hop[kLcMaxHops];  // [n, F] hop matrices, box [1, 32]
+    CUtensorMap y[kLcMaxHops];    // [batch_size, hidden] outputs, box [32, 32]
+    CUtensorMap w;                // [hidden, F] weight, box [hidden, 32]
 };
 
 struct LcArgs {
@@ -61,10 +66,12 @@ struct LcArgs {
     int32_t k_chunks;      // ceil(F / 32)
     int32_t hidden;
     uint64_t relu_mask;    // bit k: apply ReLU to hop k's output
-    float* y;
-    int64_t ldy;
-    int64_t y_hop_stride;
     int32_t* error;
+    int32_t stages;        // operand stages in flight
+    uint32_t stage_stride; // bytes between stages
+    int32_t w_resident;    // the weight is loaded once into shared memory at w_off
+    uint32_t w_off;        // offsets from the 1024-byte aligned start of dynamic shared memory
+    uint32_t epi_off;
 };
 
 __device__ __forceinline__ uint32_t lc_smem_u32(const void* p) {
@@ -156,18 +163,31 @@ __device__ __forceinline__ void lc_mma_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-__device__ __forceinline__ void lc_tmem_load16(uint32_t taddr, uint32_t (&v)[16]) {
+// 32 consecutive accumulator columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void lc_tmem_load32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
         : "r"(taddr)
         : "memory");
 }
 
+// Tensor store of one [32 rows, 32 columns] box (128-byte swizzle) from shared memory; rows and
+// columns beyond the matrix are clipped by the copy engine.
+__device__ __forceinline__ void lc_tile_store(const CUtensorMap* tmap, int x0, int y0, uint32_t src) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.tile.bulk_group [%0, {%2, %3}], [%1];" ::"l"(
+                     reinterpret_cast<uint64_t>(tmap)),
+                 "r"(src), "r"(x0), "r"(y0)
+                 : "memory");
+}
+
 __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_constant__ LcMaps maps, const LcArgs a) {
     extern __shared__ unsigned char lc_smem[];
-    __shared__ __align__(8) unsigned long long bars[2 * kLcStages + 5];
+    __shared__ __align__(8) unsigned long long bars[2 * kLcMaxStages + 6];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_word;
     volatile int* abort_flag = &abort_word;
@@ -176,13 +196,14 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
     const uint32_t tiles0 = (lc_smem_u32(lc_smem) + 1023u) & ~1023u;  // operand tiles need 1024-byte alignment
     const uint32_t bar0 = lc_smem_u32(&bars[0]);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (kLcStages + s); };
-    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * kLcStages + b); };
-    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * kLcStages + 2 + b); };
-    const uint32_t drain_bar = bar0 + 8u * (2 * kLcStages + 4);
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kLcMaxStages + s); };
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * kLcMaxStages + b); };
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * kLcMaxStages + 2 + b); };
+    const uint32_t drain_bar = bar0 + 8u * (2 * kLcMaxStages + 4);
+    const uint32_t w_bar = bar0 + 8u * (2 * kLcMaxStages + 5);
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kLcStages; ++s) {
+        for (int s = 0; s < kLcMaxStages; ++s) {
             lc_mbar_init(full_bar(s), 1);
             lc_mbar_init(empty_bar(s), 1);
         }
@@ -191,6 +212,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
             lc_mbar_init(acc_empty_bar(b), 4);  // one arrival per epilogue warp
         }
         lc_mbar_init(drain_bar, 1);
+        lc_mbar_init(w_bar, 1);
         abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -206,11 +228,20 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
     const uint32_t tmem_base = tmem_slot;
 
     const int total_tiles = a.num_hops * a.tiles_m;
-    const uint32_t stage_tx = (uint32_t)(kLcABytes + a.hidden * 128);
+    const uint32_t w_chunk_bytes = (uint32_t)a.hidden * 128u;
+    const uint32_t stage_tx = a.w_resident ? (uint32_t)kLcABytes : (uint32_t)kLcABytes + w_chunk_bytes;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- producer
-        uint32_t g = 0;  // chunks issued so far, over all tiles
+        if (a.w_resident && lane == 0) {  // the whole weight, once: it stays in shared memory for every tile
+            lc_mbar_arrive_expect_tx(w_bar, (uint32_t)a.k_chunks * w_chunk_bytes);
+            for (int kc = 0; kc < a.k_chunks; ++kc)
+                lc_tile_load(tiles0 + a.w_off + (uint32_t)kc * w_chunk_bytes, &maps.w, kc * kLcChunk, 0, w_bar);
+        }
+        __syncwarp();
+        int s = 0;
+        uint32_t ph = 0;
+        uint32_t issued = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
@@ -221,57 +252,65 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
                 if (pos >= a.batch_size) pos = a.batch_size - 1;  // rows of a ragged last tile: fetched, never stored
                 r[j] = a.batch ? __ldg(a.batch + pos) : (int)pos;
             }
-            for (int kc = 0; kc < a.k_chunks; ++kc, ++g) {
-                const int s = g % kLcStages;
-                const uint32_t ph = (g / kLcStages) & 1u;
+            for (int kc = 0; kc < a.k_chunks; ++kc) {
                 if (!__all_sync(0xffffffffu, lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error))) {
                     ok = false;
                     break;
                 }
-                const uint32_t a_dst = tiles0 + (uint32_t)s * kLcStageBytes;
+                const uint32_t a_dst = tiles0 + (uint32_t)s * a.stage_stride;
                 if (lane == 0) lc_mbar_arrive_expect_tx(full_bar(s), stage_tx);
                 __syncwarp();
                 lc_gather4(a_dst + 512u * lane, &maps.hop[hop], kc * kLcChunk, r[0], r[1], r[2], r[3], full_bar(s));
-                if (lane == 0) lc_tile_load(a_dst + kLcABytes, &maps.w, kc * kLcChunk, 0, full_bar(s));
+                if (!a.w_resident && lane == 0) lc_tile_load(a_dst + kLcABytes, &maps.w, kc * kLcChunk, 0, full_bar(s));
+                ++issued;
+                if (++s == a.stages) {
+                    s = 0;
+                    ph ^= 1u;
+                }
             }
         }
         // copies still in flight land in this CTA's shared memory: wait for them before leaving
-        const uint32_t issued = g;
-        for (int s = 0; s < kLcStages; ++s) {
-            if (issued <= (uint32_t)s) continue;
-            const uint32_t last = ((issued - 1 - s) / kLcStages) * kLcStages + s;  // last chunk that used stage s
-            const uint32_t ph = (last / kLcStages) & 1u;
+        for (int back = 0; back < a.stages && (uint32_t)back < issued; ++back) {
+            if (--s < 0) {  // walk the stages backwards from the last one filled
+                s = a.stages - 1;
+                ph ^= 1u;
+            }
             for (uint32_t i = 0; i < kLcSpinLimit; ++i)
                 if (lc_mbar_try_wait(full_bar(s), ph)) break;
         }
+        if (a.w_resident)
+            for (uint32_t i = 0; i < kLcSpinLimit; ++i)
+                if (lc_mbar_try_wait(w_bar, 0)) break;
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc = lc_instr_desc(a.hidden);
-            uint32_t g = 0;
-            int it = 0;
-            bool ok = true;
+            int s = 0, it = 0;
+            uint32_t ph = 0;
+            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error);
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
                 const int buf = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
                 if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + (uint32_t)buf * kLcMaxHidden;
-                for (int kc = 0; kc < a.k_chunks; ++kc, ++g) {
-                    const int s = g % kLcStages;
-                    const uint32_t ph = (g / kLcStages) & 1u;
+                for (int kc = 0; kc < a.k_chunks; ++kc) {
                     if (!lc_wait(full_bar(s), ph, abort_flag, a.error)) {
                         ok = false;
                         break;
                     }
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t a_src = tiles0 + (uint32_t)s * kLcStageBytes;
-                    const uint32_t b_src = a_src + kLcABytes;
+                    const uint32_t a_src = tiles0 + (uint32_t)s * a.stage_stride;
+                    const uint32_t b_src = a.w_resident ? tiles0 + a.w_off + (uint32_t)kc * w_chunk_bytes : a_src + kLcABytes;
 #pragma unroll
                     for (int j = 0; j < kLcChunk / 8; ++j)
                         lc_mma_tf32(tmem_d, lc_operand_desc(a_src + 32u * j), lc_operand_desc(b_src + 32u * j), idesc,
                                     (kc | j) != 0);
                     lc_mma_commit(empty_bar(s));  // the stage is free once these MMAs have read it
+                    if (++s == a.stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
                 }
                 if (ok) lc_mma_commit(acc_full_bar(buf));
             }
@@ -284,6 +323,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
     } else {
         // ---------------------------------------------------------------- epilogue
         const int q = warp & 3;  // tensor-memory lanes 32q .. 32q+31 belong to this warp
+        const uint32_t stage_buf = tiles0 + a.epi_off + (uint32_t)(warp - 2) * (2u * kLcEpiBytes);
+        uint32_t stored = 0;  // boxes this warp has handed to the copy engine
         int it = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {
             const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
@@ -291,33 +332,43 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
             if (!__all_sync(0xffffffffu, lc_wait(acc_full_bar(buf), acc_ph, abort_flag, a.error))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const int64_t pos = (int64_t)mt * kLcTileM + 32 * q + lane;
             const bool relu = (a.relu_mask >> hop) & 1u;
-            float* yrow = a.y + (int64_t)hop * a.y_hop_stride + pos * a.ldy;
             const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)buf * kLcMaxHidden;
-            for (int c0 = 0; c0 < a.hidden; c0 += 16) {
-                uint32_t v[16];
-                lc_tmem_load16(taddr + (uint32_t)c0, v);
+            for (int c0 = 0; c0 < a.hidden; c0 += 32, ++stored) {
+                uint32_t v[32];
+                lc_tmem_load32(taddr + (uint32_t)c0, v);
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (pos < a.batch_size) {
+                const uint32_t box = stage_buf + (stored & 1u) * kLcEpiBytes;
+                // the store that used this buffer two boxes ago must have read it
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                __syncwarp();
 #pragma unroll
-                    for (int j = 0; j < 16; j += 4) {
-                        float4 o = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]),
-                                               __uint_as_float(v[j + 3]));
-                        if (relu) {
-                            o.x = fmaxf(o.x, 0.f);
-                            o.y = fmaxf(o.y, 0.f);
-                            o.z = fmaxf(o.z, 0.f);
-                            o.w = fmaxf(o.w, 0.f);
-                        }
-                        *reinterpret_cast<float4*>(yrow + c0 + j) = o;
+                for (int j = 0; j < 8; ++j) {
+                    float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
+                                           __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    if (relu) {
+                        o.x = fmaxf(o.x, 0.f);
+                        o.y = fmaxf(o.y, 0.f);
+                        o.z = fmaxf(o.z, 0.f);
+                        o.w = fmaxf(o.w, 0.f);
                     }
+                    // row `lane` of the box, 16-byte piece j, in the 128-byte swizzle (no bank conflicts)
+                    const uint32_t dst = box + 128u * lane + ((uint32_t)(j ^ (lane & 7)) << 4);
+                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y), "f"(o.z), "f"(o.w)
+                                 : "memory");
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) {
+                    lc_tile_store(&maps.y[hop], c0, mt * kLcTileM + 32 * q, box);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
             asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
             __syncwarp();
             if (lane == 0) lc_mbar_arrive(acc_empty_bar(buf));
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
         __syncwarp();
     }
 
@@ -388,27 +439,42 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
     GNNPRE_CUDA(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    const size_t smem = (size_t)kLcStages * kLcStageBytes + 1024;
+    // Shared memory: [operand stages][resident weight, when it fits][4 warps x 2 output boxes], after the
+    // 1024-byte alignment slack.
+    const int32_t k_chunks = (int32_t)((feat_dim + kLcChunk - 1) / kLcChunk);
+    const int64_t w_bytes = (int64_t)k_chunks * hidden * 128;
+    const bool resident = w_bytes <= kLcResidentMax;
+    const uint32_t stage_stride = resident ? (uint32_t)kLcABytes : (uint32_t)(kLcABytes + hidden * 128);
+    const int32_t stages =
+        (int32_t)std::min<int64_t>(kLcMaxStages, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
+    const uint32_t w_off = (uint32_t)stages * stage_stride;
+    const uint32_t epi_off = w_off + (resident ? (uint32_t)w_bytes : 0u);
+    const size_t smem = 1024 + (size_t)epi_off + 4 * 2 * kLcEpiBytes;
     GNNPRE_CUDA(cudaFuncSetAttribute(k_lc_first_layer, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
     LcMaps maps;
     GNNPRE_TRY(encode_map_2d(Wt, feat_dim, hidden, ldw, kLcChunk, (int)hidden, &maps.w));
-    for (int32_t k0 = 0; k0 < num_hops; k0 += kLcMaxHops) {  // at most kLcMaxHops tensor maps ride in one launch
+    for (int32_t k0 = 0; k0 < num_hops; k0 += kLcMaxHops) {  // at most kLcMaxHops hop matrices ride in one launch
         const int32_t kn = std::min<int32_t>(kLcMaxHops, num_hops - k0);
-        for (int32_t k = 0; k < kLcMaxHops; ++k)
-            GNNPRE_TRY(encode_map_2d(hops[k0 + std::min(k, kn - 1)], feat_dim, n, ldh, kLcChunk, 1, &maps.hop[k]));
+        for (int32_t k = 0; k < kLcMaxHops; ++k) {
+            const int32_t kk = k0 + std::min(k, kn - 1);
+            GNNPRE_TRY(encode_map_2d(hops[kk], feat_dim, n, ldh, kLcChunk, 1, &maps.hop[k]));
+            GNNPRE_TRY(encode_map_2d(Y + (int64_t)kk * y_hop_stride, hidden, batch_size, ldy, 32, 32, &maps.y[k]));
+        }
         LcArgs a;
         a.batch = batch;
         a.batch_size = batch_size;
         a.num_hops = kn;
         a.tiles_m = (int32_t)tiles_m;
-        a.k_chunks = (int32_t)((feat_dim + kLcChunk - 1) / kLcChunk);
+        a.k_chunks = k_chunks;
         a.hidden = (int32_t)hidden;
         a.relu_mask = relu_mask >> k0;
-        a.y = Y + (int64_t)k0 * y_hop_stride;
-        a.ldy = ldy;
-        a.y_hop_stride = y_hop_stride;
         a.error = error_flag;
+        a.stages = stages;
+        a.stage_stride = stage_stride;
+        a.w_resident = resident ? 1 : 0;
+        a.w_off = w_off;
+        a.epi_off = epi_off;
         const int64_t total = (int64_t)kn * tiles_m;
         const unsigned grid = (unsigned)std::min<int64_t>(num_sms, total);
         k_lc_first_layer<<<grid, kLcThreads, smem, st>>>(maps, a);
