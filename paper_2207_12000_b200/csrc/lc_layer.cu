@@ -11,8 +11,8 @@
 //   warp 1   one lane issues tcgen05.mma (kind::tf32, M = 128, N = hidden, K = 8 per instruction,
 //            operands read from shared memory through swizzled K-major descriptors, fp32 accumulator
 //            in tensor memory) and hands stages back with tcgen05.commit on the `empty` mbarrier.
-//   warps 2-5  epilogue.  Each warp owns one quarter of the accumulator's 128 lanes, pulls it out of
-//            tensor memory with tcgen05.ld 32 columns at a time, applies ReLU where asked, lays the
+//   warps 2-9  epilogue.  Two warps share each quarter of the accumulator's 128 lanes (even and odd
+//            column boxes); a warp pulls its part out of tensor memory with tcgen05.ld 32 columns at a time, applies ReLU where asked, lays the
 //            [32, 32] box down in shared memory (128-byte swizzle, conflict-free) and hands it to the
 //            copy engine as a tensor store, which writes whole lines and clips the ragged edges.
 //
@@ -46,7 +46,7 @@ constexpr int kLcResidentMax = 128 * 1024;        // largest weight kept in shar
 constexpr int kLcEpiBytes = 32 * 128;             // one [32, 32] fp32 output box
 constexpr int kLcMaxHidden = 256;                 // N of one MMA, columns of one accumulator buffer
 constexpr int kLcABytes = kLcTileM * 128;         // 16 KB
-constexpr int kLcThreads = 192;
+constexpr int kLcThreads = 320;                    // producer warp, MMA warp, eight epilogue warps
 constexpr int kLcMaxHops = 8;                     // hop matrices (tensor maps) per launch
 constexpr uint32_t kLcTmemCols = 512;
 constexpr uint32_t kLcSuspendNs = 20000;          // a failed poll parks the warp for up to this long
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         }
         for (int b = 0; b < 2; ++b) {
             lc_mbar_init(acc_full_bar(b), 1);
-            lc_mbar_init(acc_empty_bar(b), 4);  // one arrival per epilogue warp
+            lc_mbar_init(acc_empty_bar(b), 8);  // one arrival per epilogue warp
         }
         lc_mbar_init(drain_bar, 1);
         lc_mbar_init(w_bar, 1);
@@ -322,9 +322,12 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         __syncwarp();
     } else {
         // ---------------------------------------------------------------- epilogue
-        const int q = warp & 3;  // tensor-memory lanes 32q .. 32q+31 belong to this warp
-        const uint32_t stage_buf = tiles0 + a.epi_off + (uint32_t)(warp - 2) * (2u * kLcEpiBytes);
-        uint32_t stored = 0;  // boxes this warp has handed to the copy engine
+        // Two warps per quarter of the accumulator's lanes: warps 2-5 take the even 32-column boxes,
+        // warps 6-9 the odd ones.
+        const int q = warp & 3;  // tensor-memory lanes 32q .. 32q+31 are the ones this warp may read
+        const int half = (warp - 2) >> 2;
+        const uint32_t box = tiles0 + a.epi_off + (uint32_t)(warp - 2) * kLcEpiBytes;
+        const int boxes = (a.hidden + 31) / 32;
         int it = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {
             const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
@@ -334,18 +337,20 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             const bool relu = (a.relu_mask >> hop) & 1u;
             const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)buf * kLcMaxHidden;
-            for (int c0 = 0; c0 < a.hidden; c0 += 32, ++stored) {
-                uint32_t v[32];
-                lc_tmem_load32(taddr + (uint32_t)c0, v);
+            // the read of box i + 2 is in flight while box i is written out
+            uint32_t v[2][32];
+            if (half < boxes) lc_tmem_load32(taddr + 32u * half, v[0]);
+#pragma unroll 2
+            for (int i = half, u = 0; i < boxes; i += 2, u ^= 1) {
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                const uint32_t box = stage_buf + (stored & 1u) * kLcEpiBytes;
-                // the store that used this buffer two boxes ago must have read it
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                if (i + 2 < boxes) lc_tmem_load32(taddr + 32u * (i + 2), v[u ^ 1]);
+                // the previous store must have read the staging box before it is overwritten
+                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
                 __syncwarp();
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    float4 o = make_float4(__uint_as_float(v[4 * j]), __uint_as_float(v[4 * j + 1]),
-                                           __uint_as_float(v[4 * j + 2]), __uint_as_float(v[4 * j + 3]));
+                    float4 o = make_float4(__uint_as_float(v[u][4 * j]), __uint_as_float(v[u][4 * j + 1]),
+                                           __uint_as_float(v[u][4 * j + 2]), __uint_as_float(v[u][4 * j + 3]));
                     if (relu) {
                         o.x = fmaxf(o.x, 0.f);
                         o.y = fmaxf(o.y, 0.f);
@@ -360,7 +365,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) {
-                    lc_tile_store(&maps.y[hop], c0, mt * kLcTileM + 32 * q, box);
+                    lc_tile_store(&maps.y[hop], 32 * i, mt * kLcTileM + 32 * q, box);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             }
@@ -439,7 +444,7 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
     GNNPRE_CUDA(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
     cudaStream_t st = static_cast<cudaStream_t>(stream);
 
-    // Shared memory: [operand stages][resident weight, when it fits][4 warps x 2 output boxes], after the
+    // Shared memory: [operand stages][resident weight, when it fits][8 warps x 1 output box], after the
     // 1024-byte alignment slack.
     const int32_t k_chunks = (int32_t)((feat_dim + kLcChunk - 1) / kLcChunk);
     const int64_t w_bytes = (int64_t)k_chunks * hidden * 128;
@@ -449,7 +454,7 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
         (int32_t)std::min<int64_t>(kLcMaxStages, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
     const uint32_t w_off = (uint32_t)stages * stage_stride;
     const uint32_t epi_off = w_off + (resident ? (uint32_t)w_bytes : 0u);
-    const size_t smem = 1024 + (size_t)epi_off + 4 * 2 * kLcEpiBytes;
+    const size_t smem = 1024 + (size_t)epi_off + 8 * kLcEpiBytes;
     GNNPRE_CUDA(cudaFuncSetAttribute(k_lc_first_layer, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
     LcMaps maps;
