@@ -4,14 +4,18 @@
 // This is the one dense contraction next to the aggregation path, so it runs on the 5th-generation
 // tensor cores: a persistent, warp-specialised kernel with one CTA per SM.
 //
-//   warp 0   producer.  Per K-chunk of 32 features it gathers the 128 batch rows of the tile straight
-//            out of the hop matrix with 32 tile::gather4 tensor copies (one per lane, four rows each,
-//            128-byte swizzle) and fetches the matching [hidden, 32] chunk of the weight with one
-//            tiled tensor copy; completion is counted in bytes on the stage's `full` mbarrier.
-//   warp 1   one lane issues tcgen05.mma (kind::tf32, M = 128, N = hidden, K = 8 per instruction,
+//   warps 0-3  producers.  Per K-chunk of 32 features they gather the 128 batch rows of the tile straight
+//            out of the hop matrix into the 128-byte-swizzled operand layout with 16-byte asynchronous
+//            copies (cp.async: no registers, zero fill past the last feature and for rows outside the
+//            batch), keep three chunks in flight beyond the one they announce, and arrive on the stage's
+//            `full` mbarrier after a proxy fence.  (Tensor copies in tile::gather4 mode were measured
+//            first: at 128 bytes per gathered row the copy engine's per-row rate, about 95 rows per
+//            microsecond and SM, capped the kernel at 60 % of what the output stores alone sustain.)
+//            The weight travels by tiled tensor copies, counted in bytes on an mbarrier.
+//   warp 4   one lane issues tcgen05.mma (kind::tf32, M = 128, N = hidden, K = 8 per instruction,
 //            operands read from shared memory through swizzled K-major descriptors, fp32 accumulator
 //            in tensor memory) and hands stages back with tcgen05.commit on the `empty` mbarrier.
-//   warps 2-9  epilogue.  Two warps share each quarter of the accumulator's 128 lanes (even and odd
+//   warps 5-12  epilogue.  Two warps share each quarter of the accumulator's 128 lanes (even and odd
 //            column boxes); a warp pulls its part out of tensor memory with tcgen05.ld 32 columns at a time, applies ReLU where asked, lays the
 //            [32, 32] box down in shared memory (128-byte swizzle, conflict-free) and hands it to the
 //            copy engine as a tensor store, which writes whole lines and clips the ragged edges.
@@ -26,7 +30,7 @@
 // and accumulates in fp32.
 //
 // Every wait is bounded.  A wait that runs out raises the CTA's abort flag and the caller's error
-// word; every role then leaves its loop, the producer waits (bounded) for the copies it still has in
+// word; every role then leaves its loop, the producers wait for the copies they still have in
 // flight, the MMA lane waits (bounded) for the tensor core to drain, and tensor memory is freed.
 #include <algorithm>
 #include <cstdint>
@@ -41,24 +45,31 @@ namespace {
 constexpr int kLcTileM = 128;                     // batch rows per tile = accumulator lanes
 constexpr int kLcChunk = 32;                      // features per stage: 32 fp32 = one 128-byte swizzle row
 constexpr int kLcMaxStages = 8;
+constexpr int kLcLookahead = 3;                   // chunks a producer thread keeps in flight beyond the one it announces
 constexpr int kLcPipeBytes = 192 * 1024;          // operand stages plus, when it fits, the resident weight
 constexpr int kLcResidentMax = 128 * 1024;        // largest weight kept in shared memory for the whole launch
 constexpr int kLcEpiBytes = 32 * 128;             // one [32, 32] fp32 output box
 constexpr int kLcMaxHidden = 256;                 // N of one MMA, columns of one accumulator buffer
 constexpr int kLcABytes = kLcTileM * 128;         // 16 KB
-constexpr int kLcThreads = 320;                    // producer warp, MMA warp, eight epilogue warps
-constexpr int kLcMaxHops = 8;                     // hop matrices (tensor maps) per launch
+constexpr int kLcProducerWarps = 4;
+constexpr int kLcProducerThreads = 32 * kLcProducerWarps;
+constexpr int kLcMmaWarp = kLcProducerWarps;       // warps: 0-3 producers, 4 MMA, 5-12 epilogue
+constexpr int kLcThreads = 32 * (kLcProducerWarps + 1 + 8);
+constexpr int kLcMaxHops = 8;                     // hop matrices per launch
 constexpr uint32_t kLcTmemCols = 512;
 constexpr uint32_t kLcSuspendNs = 20000;          // a failed poll parks the warp for up to this long
 constexpr uint32_t kLcSpinLimit = 50000;          // polls before a wait gives up (about a second)
 
 struct LcMaps {
-    CUtensorMap hop[kLcMaxHops];  // [n, F] hop matrices, box [1, 32]
     CUtensorMap y[kLcMaxHops];    // [batch_size, hidden] outputs, box [32, 32]
     CUtensorMap w;                // [hidden, F] weight, box [hidden, 32]
 };
 
 struct LcArgs {
+    const float* hop[kLcMaxHops];  // [n, F] hop matrices, leading dimension ldh
+    int64_t ldh;
+    int64_t n;
+    int32_t feat_dim;
     const int32_t* batch;  // row of the hop matrices for each batch position, or nullptr = identity
     int64_t batch_size;
     int32_t num_hops;
@@ -114,13 +125,10 @@ __device__ __forceinline__ bool lc_wait(uint32_t bar, uint32_t parity, volatile 
     return false;
 }
 
-__device__ __forceinline__ void lc_gather4(uint32_t dst, const CUtensorMap* tmap, int x0, int r0, int r1, int r2, int r3,
-                                           uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];" ::"r"(dst),
-        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(bar), "r"(x0), "r"(r0), "r"(r1), "r"(r2), "r"(r3)
-        : "memory");
+// 16 bytes global -> shared without passing through registers; only the first src_bytes (0..16) are
+// read, the rest of the 16 bytes is written as zeros.
+__device__ __forceinline__ void lc_copy16(uint32_t dst, const float* src, uint32_t src_bytes) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 
 __device__ __forceinline__ void lc_tile_load(uint32_t dst, const CUtensorMap* tmap, int x0, int y0, uint32_t bar) {
@@ -204,7 +212,9 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kLcMaxStages; ++s) {
-            lc_mbar_init(full_bar(s), 1);
+            // every producer thread arrives once its copies have landed; a streamed weight chunk adds
+            // one arrival that carries the chunk's byte count
+            lc_mbar_init(full_bar(s), kLcProducerThreads + (a.w_resident ? 0 : 1));
             lc_mbar_init(empty_bar(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -216,7 +226,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kLcMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lc_smem_u32(&tmem_slot)),
                      "r"(kLcTmemCols)
                      : "memory");
@@ -229,59 +239,97 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 
     const int total_tiles = a.num_hops * a.tiles_m;
     const uint32_t w_chunk_bytes = (uint32_t)a.hidden * 128u;
-    const uint32_t stage_tx = a.w_resident ? (uint32_t)kLcABytes : (uint32_t)kLcABytes + w_chunk_bytes;
 
-    if (warp == 0) {
-        // ---------------------------------------------------------------- producer
-        if (a.w_resident && lane == 0) {  // the whole weight, once: it stays in shared memory for every tile
+    if (warp < kLcProducerWarps) {
+        // ---------------------------------------------------------------- producers
+        const int pt = threadIdx.x;  // 0..127
+        if (a.w_resident && pt == 0) {  // the whole weight, once: it stays in shared memory for every tile
             lc_mbar_arrive_expect_tx(w_bar, (uint32_t)a.k_chunks * w_chunk_bytes);
             for (int kc = 0; kc < a.k_chunks; ++kc)
                 lc_tile_load(tiles0 + a.w_off + (uint32_t)kc * w_chunk_bytes, &maps.w, kc * kLcChunk, 0, w_bar);
         }
-        __syncwarp();
-        int s = 0;
+        // Eight consecutive lanes copy the eight 16-byte pieces of one row's chunk (128 contiguous bytes);
+        // a warp instruction covers four rows, a thread eight rows of its warp's 32.
+        const int piece = lane & 7;
+        const int row0 = 32 * warp + (lane >> 3);            // this thread's rows: row0 + 4 i, i < 8
+        int s = 0;           // stage the next chunk goes to
         uint32_t ph = 0;
-        uint32_t issued = 0;
+        int s_done = 0;      // stage whose copies are announced next
+        uint32_t issued = 0, announced = 0;
         bool ok = true;
         for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x) {
             const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
-            int r[4];
+            const float* src_row[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                int64_t pos = (int64_t)mt * kLcTileM + 4 * lane + j;
-                if (pos >= a.batch_size) pos = a.batch_size - 1;  // rows of a ragged last tile: fetched, never stored
-                r[j] = a.batch ? __ldg(a.batch + pos) : (int)pos;
+            for (int i = 0; i < 8; ++i) {
+                const int64_t pos = (int64_t)mt * kLcTileM + row0 + 4 * i;
+                int64_t r = -1;
+                if (pos < a.batch_size) r = a.batch ? (int64_t)__ldg(a.batch + pos) : pos;
+                // rows past the batch and indices outside the matrix are read as zeros (no bytes fetched)
+                src_row[i] = (r >= 0 && r < a.n) ? a.hop[hop] + r * a.ldh : nullptr;
             }
             for (int kc = 0; kc < a.k_chunks; ++kc) {
-                if (!__all_sync(0xffffffffu, lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error))) {
+                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error)) {
                     ok = false;
                     break;
                 }
+                const int col = kc * kLcChunk + 4 * piece;
+                const int left = a.feat_dim - col;                     // valid floats from col on
+                const uint32_t bytes = left >= 4 ? 16u : left > 0 ? 4u * left : 0u;
                 const uint32_t a_dst = tiles0 + (uint32_t)s * a.stage_stride;
-                if (lane == 0) lc_mbar_arrive_expect_tx(full_bar(s), stage_tx);
-                __syncwarp();
-                lc_gather4(a_dst + 512u * lane, &maps.hop[hop], kc * kLcChunk, r[0], r[1], r[2], r[3], full_bar(s));
-                if (!a.w_resident && lane == 0) lc_tile_load(a_dst + kLcABytes, &maps.w, kc * kLcChunk, 0, full_bar(s));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    // row (row0 + 4 i) of the tile, 16-byte piece `piece`, in the 128-byte swizzle
+                    const int row = row0 + 4 * i;
+                    const uint32_t dst = a_dst + 128u * row + ((uint32_t)(piece ^ (row & 7)) << 4);
+                    const bool live = src_row[i] != nullptr && bytes != 0;
+                    lc_copy16(dst, live ? src_row[i] + col : a.hop[hop], live ? bytes : 0u);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                if (!a.w_resident && pt == 0) {
+                    lc_mbar_arrive_expect_tx(full_bar(s), w_chunk_bytes);
+                    lc_tile_load(a_dst + kLcABytes, &maps.w, kc * kLcChunk, 0, full_bar(s));
+                }
                 ++issued;
                 if (++s == a.stages) {
                     s = 0;
                     ph ^= 1u;
                 }
+                if (issued - announced > (uint32_t)kLcLookahead) {
+                    // all but the newest kLcLookahead groups have landed: hand the oldest to the MMA warp
+                    asm volatile("cp.async.wait_group %0;" ::"n"(kLcLookahead) : "memory");
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    lc_mbar_arrive(full_bar(s_done));
+                    ++announced;
+                    if (++s_done == a.stages) s_done = 0;
+                }
             }
         }
-        // copies still in flight land in this CTA's shared memory: wait for them before leaving
-        for (int back = 0; back < a.stages && (uint32_t)back < issued; ++back) {
-            if (--s < 0) {  // walk the stages backwards from the last one filled
-                s = a.stages - 1;
-                ph ^= 1u;
-            }
-            for (uint32_t i = 0; i < kLcSpinLimit; ++i)
-                if (lc_mbar_try_wait(full_bar(s), ph)) break;
+        // the tail: everything still in flight lands, then the remaining chunks are announced
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        while (announced < issued) {
+            lc_mbar_arrive(full_bar(s_done));
+            ++announced;
+            if (++s_done == a.stages) s_done = 0;
         }
-        if (a.w_resident)
-            for (uint32_t i = 0; i < kLcSpinLimit; ++i)
-                if (lc_mbar_try_wait(w_bar, 0)) break;
-    } else if (warp == 1) {
+        // tensor copies of the weight land in this CTA's shared memory: wait for them before leaving
+        if (pt == 0) {
+            if (a.w_resident) {
+                for (uint32_t i = 0; i < kLcSpinLimit; ++i)
+                    if (lc_mbar_try_wait(w_bar, 0)) break;
+            } else {
+                for (int back = 0; back < a.stages && (uint32_t)back < issued; ++back) {
+                    if (--s < 0) {  // walk the stages backwards from the last one filled
+                        s = a.stages - 1;
+                        ph ^= 1u;
+                    }
+                    for (uint32_t i = 0; i < kLcSpinLimit; ++i)
+                        if (lc_mbar_try_wait(full_bar(s), ph)) break;
+                }
+            }
+        }
+    } else if (warp == kLcMmaWarp) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
             const uint32_t idesc = lc_instr_desc(a.hidden);
@@ -322,11 +370,12 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         __syncwarp();
     } else {
         // ---------------------------------------------------------------- epilogue
-        // Two warps per quarter of the accumulator's lanes: warps 2-5 take the even 32-column boxes,
-        // warps 6-9 the odd ones.
-        const int q = warp & 3;  // tensor-memory lanes 32q .. 32q+31 are the ones this warp may read
-        const int half = (warp - 2) >> 2;
-        const uint32_t box = tiles0 + a.epi_off + (uint32_t)(warp - 2) * kLcEpiBytes;
+        // Two warps per quarter of the accumulator's lanes: the first four epilogue warps take the even
+        // 32-column boxes, the last four the odd ones.
+        const int ew = warp - kLcMmaWarp - 1;  // 0..7
+        const int q = warp & 3;                // tensor-memory lanes 32q .. 32q+31 are the ones this warp may read
+        const int half = ew >> 2;
+        const uint32_t box = tiles0 + a.epi_off + (uint32_t)ew * kLcEpiBytes;
         const int boxes = (a.hidden + 31) / 32;
         int it = 0;
         for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {
@@ -379,7 +428,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kLcMmaWarp) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kLcTmemCols) : "memory");
     }
@@ -461,12 +510,15 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
     GNNPRE_TRY(encode_map_2d(Wt, feat_dim, hidden, ldw, kLcChunk, (int)hidden, &maps.w));
     for (int32_t k0 = 0; k0 < num_hops; k0 += kLcMaxHops) {  // at most kLcMaxHops hop matrices ride in one launch
         const int32_t kn = std::min<int32_t>(kLcMaxHops, num_hops - k0);
+        LcArgs a;
         for (int32_t k = 0; k < kLcMaxHops; ++k) {
             const int32_t kk = k0 + std::min(k, kn - 1);
-            GNNPRE_TRY(encode_map_2d(hops[kk], feat_dim, n, ldh, kLcChunk, 1, &maps.hop[k]));
+            a.hop[k] = hops[kk];
             GNNPRE_TRY(encode_map_2d(Y + (int64_t)kk * y_hop_stride, hidden, batch_size, ldy, 32, 32, &maps.y[k]));
         }
-        LcArgs a;
+        a.ldh = ldh;
+        a.n = n;
+        a.feat_dim = (int32_t)feat_dim;
         a.batch = batch;
         a.batch_size = batch_size;
         a.num_hops = kn;
