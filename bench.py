@@ -49,6 +49,10 @@ def parse():
     ap.add_argument("--op", type=int, default=-1, help="override the workload's operator (sweeps)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--budget-gb", type=float, default=0.0, help="device-memory budget B_GPU of the streamed plan (0 = free memory)")
+    ap.add_argument("--stage", default="aggregate", choices=["aggregate", "lc"],
+                    help="aggregate: the K-hop precomputation (the headline); lc: the first dense stage of an LC model "
+                         "(Eq. 9) over the precomputed hops, every row once in a seeded random order")
+    ap.add_argument("--hidden", type=int, default=256, help="hidden width of --stage lc")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -121,6 +125,26 @@ def profiled_traffic(workload_name):
     for f in ("propagate.cu", "segments_tma.cuh"):
         cur.update(open(os.path.join(ROOT, "paper_2207_12000_b200", "csrc", f), "rb").read())
     return int(t.group(1)) if cur.hexdigest() == h.group(1) else None
+
+
+def profiled_traffic_lc(rows_per_launch):
+    """DRAM bytes per launch of k_lc_first_layer: the committed ncu figure of a smaller case scaled by gathered
+    rows (traffic is proportional to them), or None when the kernel source has changed since the capture."""
+    import hashlib
+    import re
+    path = os.path.join(ROOT, "profiles", "k_lc_first_layer_c4_quarter_scale_dram.md")
+    if not os.path.exists(path):
+        return None
+    text = open(path).read()
+    t = re.search(r"traffic_bytes_per_launch:\s*(\d+)", text)
+    r = re.search(r"rows_per_launch:\s*(\d+)", text)
+    h = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
+    if not t or not r or not h:
+        return None
+    src = open(os.path.join(ROOT, "paper_2207_12000_b200", "csrc", "lc_layer.cu"), "rb").read()
+    if hashlib.sha256(src).hexdigest() != h.group(1):
+        return None
+    return int(round(int(t.group(1)) * rows_per_launch / int(r.group(1))))
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
@@ -207,6 +231,85 @@ def workload_config(w, g, info):
     return cfg
 
 
+def run_lc_stage(args, w):
+    """--stage lc: Y_k = act(X_k[batch] W_1) for the K precomputed hops of the workload (Eq. 9's first dense
+    stage; hidden width and ReLU from the paper's settings).  A step is one call over all n rows in a seeded
+    random order (one epoch's worth of mini-batches); the 4096-row mini-batch is timed beside it."""
+    from paper_2207_12000_b200 import binding as B  # fails loudly if the CUDA library is missing
+    torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        raise SystemExit("--stage lc is a single-GPU measurement")
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    K, F, H, n = w.hops, w.feat_dim, args.hidden, g.n
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps)
+    hops, _ = B.gnnpre_propagate(plan, X, K)
+    plan.close()
+    del X
+    Wt = gi.normal_matrix(H, F, w.seed + 77, device="cuda") / float(np.sqrt(F))
+    order = torch.from_numpy(np.random.default_rng(w.seed).permutation(n).astype(np.int32)).cuda()
+    relu_mask = (1 << K) - 2  # sigma on every term that has another layer after it (k >= 2 in Eq. 9)
+    Y = torch.empty((K, n, H), dtype=torch.float32, device="cuda")
+    flag_check = B.gnnpre_lc_first_layer(hops, order[:4096], Wt, relu_mask=relu_mask)  # synchronising call: error word read
+    del flag_check
+    stream = torch.cuda.current_stream()
+
+    def timed(batch, out, steps, warmup):
+        for _ in range(warmup):
+            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, out=out, check=False)
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        ev[0].record(stream)
+        for i in range(steps):
+            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, out=out, check=False)
+            ev[i + 1].record(stream)
+        torch.cuda.synchronize()
+        return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+    with ClockSampler(torch.cuda.current_device()) as sampler:  # the same kernel runs in all three timings
+        ms = timed(order, Y, args.steps, max(3, args.warmup))
+        in_order = timed(None, Y, args.steps, 3)
+        mini = timed(order[:4096], Y[:, :4096], 200, 5)
+        t_end = time.perf_counter() + 1.5  # untimed: the same calls, long enough for the clock sampler to see the load
+        while time.perf_counter() < t_end:
+            timed(order, Y, 20, 0)
+    clocks = sampler.summary()
+    total_ms = float(sum(ms))
+    ms_step = total_ms / args.steps
+    elems = K * n * H
+    peak, which = measured_peaks()
+    alg_bytes = 4 * K * n * (F + H) + 4 * H * F  # every gathered row read once, every output written once, the weight once
+    achieved = alg_bytes / (ms_step * 1e-3) / 1e9
+    line = {
+        "metric": "first dense stage of an LC model: output elems/s", "value": elems / (ms_step * 1e-3), "unit": "elems/s",
+        "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32 inputs, f32 accumulate",
+        "data": "synthetic", "stage": "lc",
+        "config": {"workload": f"{w.name}: first dense stage over the {K} hops of n={n}, F={F}; hidden={H}; all rows, seeded random order",
+                   "l2": "inputs and outputs larger than L2", "mini_batch_4096_ms": float(np.median(mini)),
+                   "rows_in_order_ms": float(np.median(in_order)), "tflops": 2.0 * K * n * F * H / (ms_step * 1e-3) / 1e12},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": profiled_traffic_lc(K * n) if H == 256 and F == 100 else None, "peak_source": which,
+                     "algorithmic_bytes_per_launch": alg_bytes},
+        "gpu_launches": args.steps, "clocks": clocks, "e2e": None,
+    }
+    if not args.no_cpu_baseline:
+        import oracle as orc
+        hop0 = hops[0].cpu().numpy()
+        Wt_np = Wt.cpu().numpy()
+        rows = 2048
+        t0 = time.perf_counter()
+        orc.lc_first_layer(hop0, order[:rows].cpu().numpy(), Wt_np, relu=True)
+        t = time.perf_counter() - t0
+        rows2 = int(max(rows, min(n, rows * args.cpu_seconds / max(t, 1e-6))))
+        t0 = time.perf_counter()
+        orc.lc_first_layer(hop0, order[:rows2].cpu().numpy(), Wt_np, relu=True)
+        t = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": rows2 * H / t, "unit": "elems/s", "cores": orc.num_threads(), "kind": "oracle",
+                                "sample": f"hop 1, first {rows2} rows of the order, {t:.2f} s"}
+    print(json.dumps(line))
+
+
 def main():
     args = parse()
     w = gi.scaled(gi.WORKLOADS[args.workload], args.scale_down)
@@ -215,6 +318,9 @@ def main():
         w = dataclasses.replace(w, feat_dim=args.feat_dim or w.feat_dim, op=args.op if args.op >= 0 else w.op)
     if args.impl == "reference":
         run_reference(args, w)
+        return
+    if args.stage == "lc":
+        run_lc_stage(args, w)
         return
 
     from paper_2207_12000_b200 import binding as B  # fails loudly if the CUDA library is missing
