@@ -53,6 +53,7 @@ def parse():
                     help="aggregate: the K-hop precomputation (the headline); lc: the first dense stage of an LC model "
                          "(Eq. 9) over the precomputed hops, every row once in a seeded random order")
     ap.add_argument("--hidden", type=int, default=256, help="hidden width of --stage lc")
+    ap.add_argument("--e2e-col-slabs", type=int, default=0, help="column slabs c of the host-buffer run (0 = the library's choice)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
@@ -432,7 +433,7 @@ def main():
             else:
                 rp_e2e, ci_e2e = g.rowptr, g.colidx
             hplan = B.gnnpre_build_plan(rp_e2e, ci_e2e, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
-                                        force_col_slabs=0, segment_edges=args.segment_edges,
+                                        force_col_slabs=args.e2e_col_slabs, segment_edges=args.segment_edges,
                                         budget_bytes=int(args.budget_gb * 1e9), operands_mem=B.GNNPRE_MEM_HOST)
             for _ in range(2):
                 B.gnnpre_propagate(hplan, Xh, K, outs_h)
