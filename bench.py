@@ -296,8 +296,8 @@ def run_lc_stage(args, w):
     }
     if not args.no_cpu_baseline:
         import oracle as orc
-        hop0 = hops[0].cpu().numpy()
-        Wt_np = Wt.cpu().numpy()
+        hop0 = gi.make_features(w).numpy()  # timing only: a seeded matrix of the hop's shape, nothing from the device
+        Wt_np = gi.normal_matrix(H, F, w.seed + 77).numpy() / np.float32(np.sqrt(F))
         rows = 2048
         t0 = time.perf_counter()
         orc.lc_first_layer(hop0, order[:rows].cpu().numpy(), Wt_np, relu=True)
@@ -307,7 +307,7 @@ def run_lc_stage(args, w):
         orc.lc_first_layer(hop0, order[:rows2].cpu().numpy(), Wt_np, relu=True)
         t = time.perf_counter() - t0
         line["cpu_baseline"] = {"value": rows2 * H / t, "unit": "elems/s", "cores": orc.num_threads(), "kind": "oracle",
-                                "sample": f"hop 1, first {rows2} rows of the order, {t:.2f} s"}
+                                "sample": f"one [n, {F}] matrix, first {rows2} rows of the order, {t:.2f} s"}
     print(json.dumps(line))
 
 

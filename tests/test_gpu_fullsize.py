@@ -6,7 +6,7 @@ import torch
 
 import gnnpre_inputs as gi
 import oracle as orc
-from parity_util import TOL, backward_error, hop_error, to_np
+from parity_util import TOL, backward_error, hop_error, single_hop_of, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -22,8 +22,8 @@ def B():
 def test_config4_full_size_as_benchmarked(B):
     """2,449,029 nodes, 123.7M nnz, F=100, K=3, SAGE, 32 blocks, one launch per hop (bench.py's set-up).
     Integer plan outputs bit-exact; every hop against the full fp64 chain; sampled rows (random, the
-    highest degrees, every block-boundary row) against the exact one-hop result of the matrix the hop
-    read; the degree-weighted column sums SAGE conserves on a symmetric graph."""
+    highest degrees, every block-boundary row) against the exact one-hop result on a shared input (X_0, then
+    the oracle's previous hop in fp32); the degree-weighted column sums SAGE conserves on a symmetric graph."""
     w = gi.WORKLOADS["c4"]
     g = gi.make_graph(w, device="cuda")
     X = gi.make_features(w, device="cuda")
@@ -46,10 +46,13 @@ def test_config4_full_size_as_benchmarked(B):
     rows = np.unique(np.concatenate([rng.integers(0, g.n, 4096), np.argsort(deg.numpy())[-64:], boundary]))
     want = orc.propagate(w.op, 0.0, rp, ci, to_np(X), w.hops)
     prev = X
+    one_hop = single_hop_of(B, plan)
     for k in range(w.hops):
         got = to_np(outs[k])
         assert hop_error(got, want[k]) <= TOL
-        assert backward_error(w.op, 0.0, rp, ci, to_np(prev), got, rows) <= TOL
+        # one hop on an input both sides share: X_0, then the oracle's previous hop rounded to fp32
+        shared = to_np(X) if k == 0 else np.ascontiguousarray(want[k - 1].astype(np.float32))
+        assert backward_error(w.op, 0.0, rp, ci, shared, got if k == 0 else one_hop(shared), rows) <= TOL
         a, b_ = d @ outs[k].double(), d @ prev.double()
         scale = d @ prev.double().abs()
         assert float(((a - b_).abs() / scale).max()) <= 1e-6
@@ -92,3 +95,33 @@ def test_config5_scaled_streamed_with_budget(B):
         assert hop_error(outs[k].numpy(), want[k]) <= TOL
     plan.close()
     ref_plan.close()
+
+
+def test_first_dense_stage_at_config4_size_sampled(B):
+    """gnnpre_lc_first_layer in the launch bench.py --stage lc times: three [2,449,029 x 100] matrices, hidden 256,
+    every row once in a seeded random order (19,134 tiles per matrix, the last one ragged).  The matrices are seeded
+    synthetic stand-ins for the hops (the layer does not care where they came from); the oracle computes sampled
+    output rows one by one: random positions, the first and last tile, and the rows around every 1,000th tile edge."""
+    w = gi.WORKLOADS["c4"]
+    n, F, H, K = w.n, w.feat_dim, 256, w.hops
+    hops = [gi.normal_matrix(n, F, w.seed + 10 + k, device="cuda") for k in range(K)]
+    Wt = gi.normal_matrix(H, F, w.seed + 77, device="cuda") / float(np.sqrt(F))
+    order_np = np.random.default_rng(w.seed).permutation(n)
+    order = torch.from_numpy(order_np.astype(np.int32)).cuda()
+    relu_mask = 0b110
+    Y = B.gnnpre_lc_first_layer(hops, order, Wt, relu_mask=relu_mask)
+    rng = np.random.default_rng(11)
+    edges = np.arange(0, n, 128 * 1000)
+    pos = np.unique(np.clip(np.concatenate([rng.integers(0, n, 3000), np.arange(256), np.arange(n - 200, n),
+                                            edges - 1, edges, edges + 1]), 0, n - 1))
+    Wt_np = to_np(Wt)
+    for k in range(K):
+        want, scale = orc.lc_first_layer(to_np(hops[k]), order_np[pos], Wt_np, relu=bool((relu_mask >> k) & 1),
+                                         want_abs=True)
+        got = to_np(Y[k][torch.from_numpy(pos).cuda()]).astype(np.float64)
+        assert (np.abs(got - want) <= (2.0 ** -9 + F * 2.0 ** -23) * scale).all()
+    # properties that hold at any size: ReLU outputs are non-negative, and a second call with the identity order
+    # returns the same rows in another place, bit for bit
+    assert float(Y[1].min()) >= 0.0 and float(Y[2].min()) >= 0.0 and float(Y[0].min()) < 0.0
+    Z = B.gnnpre_lc_first_layer(hops[:1], None, Wt)
+    assert torch.equal(Z[0][order.long()[:100000]], Y[0][:100000])

@@ -12,7 +12,7 @@ import torch
 
 import gnnpre_inputs as gi
 import oracle as orc
-from parity_util import TOL, backward_error, check_all_hops, hop_error, to_np
+from parity_util import TOL, backward_error, check_all_hops, hop_error, single_hop_of, to_np
 
 pytestmark = pytest.mark.gpu
 
@@ -116,7 +116,7 @@ def run_case(B, g, op, F, K, *, b=1, c=1, seg=0, flags=0, ldx=None, ldo=None, se
     torch.cuda.synchronize()
     for o in obufs:
         assert bool((o[:, F:] == -7.0).all()), "padding columns were written"
-    worst = check_all_hops(op, EPS, rp, ci, to_np(X), outs)
+    worst = check_all_hops(op, EPS, rp, ci, to_np(X), outs, single_hop=single_hop_of(B, plan))
     plan.close()
     return worst, outs
 
@@ -202,13 +202,14 @@ def test_config3_operator_width_block_sweep(B, op, F):
         plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=w.gin_eps, force_blocks=b)
         outs, _ = B.gnnpre_propagate(plan, X, w.hops)
         torch.cuda.synchronize()
-        prev = Xn
+        one_hop = single_hop_of(B, plan)
         for k in range(w.hops):
             gk = to_np(outs[k])
             assert hop_error(gk, want[k]) <= TOL
             rows = np.random.default_rng(k).integers(0, g.n, 4096)
-            assert backward_error(op, w.gin_eps, rp, ci, prev, gk, rows) <= TOL
-            prev = gk
+            # floor-free check of one hop on an input both sides share: X_0, then the oracle's hops in fp32
+            prev = Xn if k == 0 else np.ascontiguousarray(want[k - 1].astype(np.float32))
+            assert backward_error(op, w.gin_eps, rp, ci, prev, gk if k == 0 else one_hop(prev), rows) <= TOL
         plan.close()
 
 
