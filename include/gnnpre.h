@@ -275,15 +275,23 @@ int gnnpre_hop_static(const gnnpre_csr_t* csr, int32_t op, float gin_eps, int64_
  *              (the results are then invalid).  The caller clears and reads it.
  * ldh, ldw >= feat_dim and ldy >= hidden (else INVALID_ARG); ldh, ldw, ldy, y_hop_stride multiples of 4
  * and all base pointers 16-byte aligned (else ALIGN).  feat_dim itself may be any value >= 1.
- * Arithmetic: tensor cores with tf32 inputs (the fp32 operands are read with their low 13 mantissa
- * bits ignored) and fp32 accumulation: |error| <= 2^-9 * sum_f |x||w| plus fp32 summation error.
+ * Arithmetic, by `precision`:
+ *   GNNPRE_LC_TF32    tensor cores with tf32 inputs (the fp32 operands are read with their low 13 mantissa
+ *                     bits ignored) and fp32 accumulation: |error| <= 2^-9 * sum_f |x||w| plus fp32 summation
+ *                     error.  The fastest mode.
+ *   GNNPRE_LC_TF32X3  every operand enters as the sum of two tf32 numbers (three tensor-core products per
+ *                     term, fp32 accumulation): |error| <= 2^-20 * sum_f |x||w| plus fp32 summation error,
+ *                     i.e. fp32-like accuracy.  With hidden > 128 the batch rows are fetched twice and hidden
+ *                     must be a multiple of 64 (else INVALID_ARG).
  * The work is enqueued on `stream` and the call returns without synchronising; nothing is allocated.
  * batch_size = 0 is a no-op.  UNSUPPORTED_ARCH on devices other than compute capability 10.x.
  */
+#define GNNPRE_LC_TF32 0
+#define GNNPRE_LC_TF32X3 1
 int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
                           const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw,
-                          uint64_t relu_mask, float* Y, int64_t ldy, int64_t y_hop_stride, int32_t* error_flag,
-                          void* stream);
+                          uint64_t relu_mask, int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride,
+                          int32_t* error_flag, void* stream);
 
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;

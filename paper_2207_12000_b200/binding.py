@@ -85,7 +85,7 @@ def _load() -> ctypes.CDLL:
                                      ctypes.POINTER(gnnpre_stats_t)]
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
     lib.gnnpre_lc_first_layer.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i64, i64, i64, p, i64, p, i64, i64,
-                                          ctypes.c_uint64, p, i64, i64, p, p]
+                                          ctypes.c_uint64, i32, p, i64, i64, p, p]
     lib.gnnpre_normalize.argtypes = [p, p, i32, p]
     lib.gnnpre_solve_normalisation_blocks.argtypes = [i64] * 8 + [ctypes.POINTER(i64)]
     lib.gnnpre_selftest_wait_timeout.argtypes = [p, ctypes.c_uint32, p]
@@ -238,12 +238,17 @@ def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: to
     return out
 
 
-def gnnpre_lc_first_layer(hops, batch, Wt: torch.Tensor, *, relu_mask: int = 0, out: torch.Tensor | None = None,
+GNNPRE_LC_TF32, GNNPRE_LC_TF32X3 = 0, 1
+
+
+def gnnpre_lc_first_layer(hops, batch, Wt: torch.Tensor, *, relu_mask: int = 0, precision: int = GNNPRE_LC_TF32,
+                          out: torch.Tensor | None = None,
                           concat: bool = False, check: bool = True, stream=None) -> torch.Tensor:
     """act(hops[k][batch] @ Wt.T) for every hop on the tensor cores (Eq. 9's first dense stage).
 
     hops: list of device fp32 [n, F] matrices with one common row stride; batch: device int32 row indices
     or None (all rows); Wt: device fp32 [H, F].  Returns [K, B, H], or [B, K*H] with concat=True.
+    precision: GNNPRE_LC_TF32 (tf32 operands) or GNNPRE_LC_TF32X3 (split operands, fp32-like accuracy).
     With check=True the call synchronises and raises if a device-side wait ran out."""
     K = len(hops)
     n, F = hops[0].shape
@@ -268,7 +273,7 @@ def gnnpre_lc_first_layer(hops, batch, Wt: torch.Tensor, *, relu_mask: int = 0, 
     flag = torch.zeros(1, dtype=torch.int32, device=Wt.device) if check else None
     ptrs = (ctypes.c_void_p * K)(*[h.data_ptr() for h in hops])
     _check(_lib.gnnpre_lc_first_layer(ptrs, K, n, F, hops[0].stride(0), bptr, B, Wt.data_ptr(), H, Wt.stride(0),
-                                      relu_mask, out.data_ptr(), ldy, hop_stride,
+                                      relu_mask, precision, out.data_ptr(), ldy, hop_stride,
                                       flag.data_ptr() if check else None, _stream_ptr(stream)), "gnnpre_lc_first_layer")
     if check and int(flag.item()) != 0:
         raise GnnpreError(-8, "gnnpre_lc_first_layer")

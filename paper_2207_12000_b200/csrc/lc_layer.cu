@@ -83,6 +83,12 @@ struct LcArgs {
     int32_t w_resident;    // the weight is loaded once into shared memory at w_off
     uint32_t w_off;        // offsets from the 1024-byte aligned start of dynamic shared memory
     uint32_t epi_off;
+    // the split-operand kernel only
+    const float* wt;       // [hidden, F] weight, leading dimension ldw
+    int64_t ldw;
+    int32_t halves;        // CTAs with blockIdx.x % halves == h compute output columns [h n_half, (h + 1) n_half)
+    int32_t n_half;
+    uint32_t small_off;    // offset of the low parts inside a stage
 };
 
 __device__ __forceinline__ uint32_t lc_smem_u32(const void* p) {
@@ -191,6 +197,68 @@ __device__ __forceinline__ void lc_tile_store(const CUtensorMap* tmap, int x0, i
                      reinterpret_cast<uint64_t>(tmap)),
                  "r"(src), "r"(x0), "r"(y0)
                  : "memory");
+}
+
+// Epilogue role (warps 5-12), shared by both kernels: tiles first, first + step, ...; the accumulator holds
+// n_cols columns that go to columns col0 .. col0 + n_cols of Y.  Two warps per quarter of the accumulator's
+// lanes: the first four epilogue warps take the even 32-column boxes, the last four the odd ones.
+__device__ __forceinline__ void lc_epilogue(const LcMaps& maps, const LcArgs& a, uint32_t tiles0, uint32_t tmem_base,
+                                            uint32_t acc_full0, uint32_t acc_empty0, volatile int* abort_flag, int first,
+                                            int step, int n_cols, int col0) {
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int ew = warp - kLcMmaWarp - 1;  // 0..7
+    const int q = warp & 3;                // tensor-memory lanes 32q .. 32q+31 are the ones this warp may read
+    const int half = ew >> 2;
+    const uint32_t box = tiles0 + a.epi_off + (uint32_t)ew * kLcEpiBytes;
+    const int boxes = (n_cols + 31) / 32;
+    const int total_tiles = a.num_hops * a.tiles_m;
+    int it = 0;
+    for (int t = first; t < total_tiles; t += step, ++it) {
+        const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
+        const int buf = it & 1;
+        const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+        if (!__all_sync(0xffffffffu, lc_wait(acc_full0 + 8u * buf, acc_ph, abort_flag, a.error))) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const bool relu = (a.relu_mask >> hop) & 1u;
+        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)buf * kLcMaxHidden;
+        // the read of box i + 2 is in flight while box i is written out
+        uint32_t v[2][32];
+        if (half < boxes) lc_tmem_load32(taddr + 32u * half, v[0]);
+#pragma unroll 2
+        for (int i = half, u = 0; i < boxes; i += 2, u ^= 1) {
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (i + 2 < boxes) lc_tmem_load32(taddr + 32u * (i + 2), v[u ^ 1]);
+            // the previous store must have read the staging box before it is overwritten
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+            __syncwarp();
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                float4 o = make_float4(__uint_as_float(v[u][4 * j]), __uint_as_float(v[u][4 * j + 1]),
+                                       __uint_as_float(v[u][4 * j + 2]), __uint_as_float(v[u][4 * j + 3]));
+                if (relu) {
+                    o.x = fmaxf(o.x, 0.f);
+                    o.y = fmaxf(o.y, 0.f);
+                    o.z = fmaxf(o.z, 0.f);
+                    o.w = fmaxf(o.w, 0.f);
+                }
+                // row `lane` of the box, 16-byte piece j, in the 128-byte swizzle (no bank conflicts)
+                const uint32_t dst = box + 128u * lane + ((uint32_t)(j ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y), "f"(o.z), "f"(o.w)
+                             : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+                lc_tile_store(&maps.y[hop], col0 + 32 * i, mt * kLcTileM + 32 * q, box);
+                asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+        }
+        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) lc_mbar_arrive(acc_empty0 + 8u * buf);
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
 }
 
 __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_constant__ LcMaps maps, const LcArgs a) {
@@ -370,60 +438,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         __syncwarp();
     } else {
         // ---------------------------------------------------------------- epilogue
-        // Two warps per quarter of the accumulator's lanes: the first four epilogue warps take the even
-        // 32-column boxes, the last four the odd ones.
-        const int ew = warp - kLcMmaWarp - 1;  // 0..7
-        const int q = warp & 3;                // tensor-memory lanes 32q .. 32q+31 are the ones this warp may read
-        const int half = ew >> 2;
-        const uint32_t box = tiles0 + a.epi_off + (uint32_t)ew * kLcEpiBytes;
-        const int boxes = (a.hidden + 31) / 32;
-        int it = 0;
-        for (int t = blockIdx.x; t < total_tiles; t += gridDim.x, ++it) {
-            const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
-            const int buf = it & 1;
-            const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-            if (!__all_sync(0xffffffffu, lc_wait(acc_full_bar(buf), acc_ph, abort_flag, a.error))) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const bool relu = (a.relu_mask >> hop) & 1u;
-            const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)buf * kLcMaxHidden;
-            // the read of box i + 2 is in flight while box i is written out
-            uint32_t v[2][32];
-            if (half < boxes) lc_tmem_load32(taddr + 32u * half, v[0]);
-#pragma unroll 2
-            for (int i = half, u = 0; i < boxes; i += 2, u ^= 1) {
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (i + 2 < boxes) lc_tmem_load32(taddr + 32u * (i + 2), v[u ^ 1]);
-                // the previous store must have read the staging box before it is overwritten
-                if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                __syncwarp();
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    float4 o = make_float4(__uint_as_float(v[u][4 * j]), __uint_as_float(v[u][4 * j + 1]),
-                                           __uint_as_float(v[u][4 * j + 2]), __uint_as_float(v[u][4 * j + 3]));
-                    if (relu) {
-                        o.x = fmaxf(o.x, 0.f);
-                        o.y = fmaxf(o.y, 0.f);
-                        o.z = fmaxf(o.z, 0.f);
-                        o.w = fmaxf(o.w, 0.f);
-                    }
-                    // row `lane` of the box, 16-byte piece j, in the 128-byte swizzle (no bank conflicts)
-                    const uint32_t dst = box + 128u * lane + ((uint32_t)(j ^ (lane & 7)) << 4);
-                    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y), "f"(o.z), "f"(o.w)
-                                 : "memory");
-                }
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                __syncwarp();
-                if (lane == 0) {
-                    lc_tile_store(&maps.y[hop], 32 * i, mt * kLcTileM + 32 * q, box);
-                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-                }
-            }
-            asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) lc_mbar_arrive(acc_empty_bar(buf));
-        }
-        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-        __syncwarp();
+        lc_epilogue(maps, a, tiles0, tmem_base, acc_full_bar(0), acc_empty_bar(0), abort_flag, blockIdx.x, gridDim.x,
+                    a.hidden, 0);
     }
 
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -433,6 +449,225 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kLcTmemCols) : "memory");
     }
 }
+
+// ------------------------------------------------------------------------------------------------
+// The same stage with fp32-like accuracy ("3 x tf32"): every fp32 operand is split into a high part
+// that tf32 holds exactly (low 13 mantissa bits cleared) and a low part (the remainder, again cut to
+// what tf32 holds), and  x w  ~=  xh wh + xl wh + xh wl  with fp32 accumulation; the dropped terms are
+// below 2^-21 |x||w|.  Shared memory has to hold both parts of both operands, so a CTA computes at most
+// 128 output columns: with hidden > 128, even and odd CTAs take the two halves and every batch row is
+// gathered by both (the second read mostly hits L2).  No tensor copies on the input side: the producer
+// threads bring rows of the hop matrix AND rows of the weight in with 16-byte asynchronous copies,
+// then read their own pieces back, split them and write the two parts (each thread touches only bytes
+// it copied itself, so the copy's wait_group is all the synchronisation the split needs).
+__device__ __forceinline__ void lc_split_piece(uint32_t big_addr, uint32_t small_addr) {
+    uint32_t v[4];
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(big_addr) : "memory");
+    uint32_t hi[4], lo[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        hi[j] = v[j] & 0xffffe000u;
+        lo[j] = __float_as_uint(__uint_as_float(v[j]) - __uint_as_float(hi[j])) & 0xffffe000u;  // the difference is exact
+    }
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(big_addr), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(small_addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
+}
+
+__global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __grid_constant__ LcMaps maps, const LcArgs a) {
+    extern __shared__ unsigned char lc_smem[];
+    __shared__ __align__(8) unsigned long long bars[2 * kLcMaxStages + 6];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t tiles0 = (lc_smem_u32(lc_smem) + 1023u) & ~1023u;
+    const uint32_t bar0 = lc_smem_u32(&bars[0]);
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kLcMaxStages + s); };
+    auto acc_full_bar = [&](int b) { return bar0 + 8u * (2 * kLcMaxStages + b); };
+    auto acc_empty_bar = [&](int b) { return bar0 + 8u * (2 * kLcMaxStages + 2 + b); };
+    const uint32_t drain_bar = bar0 + 8u * (2 * kLcMaxStages + 4);
+    const uint32_t w_bar = bar0 + 8u * (2 * kLcMaxStages + 5);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kLcMaxStages; ++s) {
+            lc_mbar_init(full_bar(s), kLcProducerThreads);
+            lc_mbar_init(empty_bar(s), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            lc_mbar_init(acc_full_bar(b), 1);
+            lc_mbar_init(acc_empty_bar(b), 8);
+        }
+        lc_mbar_init(drain_bar, 1);
+        lc_mbar_init(w_bar, kLcProducerThreads);
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == kLcMmaWarp) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(lc_smem_u32(&tmem_slot)),
+                     "r"(kLcTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = tmem_slot;
+
+    const int total_tiles = a.num_hops * a.tiles_m;
+    const int half = blockIdx.x % a.halves;
+    const int first = blockIdx.x / a.halves, step = gridDim.x / a.halves;
+    constexpr uint32_t kPart = kLcABytes;  // bytes of one [128 rows, 32 floats] part: 16 KB
+
+    if (warp < kLcProducerWarps) {
+        // ---------------------------------------------------------------- producers
+        const int piece = lane & 7;
+        const int row0 = 32 * warp + (lane >> 3);  // this thread's rows (of the tile and of the weight half): row0 + 4 i
+        const float* w_row[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = row0 + 4 * i;
+            w_row[i] = r < a.n_half ? a.wt + (int64_t)(half * a.n_half + r) * a.ldw : nullptr;
+        }
+        // copy this thread's pieces of chunk kc of `rows` (hop rows or weight rows) to `dst_part`
+        auto copy_chunk = [&](const auto& rows, int kc, uint32_t dst_part) {
+            const int col = kc * kLcChunk + 4 * piece;
+            const int left = a.feat_dim - col;
+            const uint32_t bytes = left >= 4 ? 16u : left > 0 ? 4u * left : 0u;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = row0 + 4 * i;
+                const uint32_t dst = dst_part + 128u * row + ((uint32_t)(piece ^ (row & 7)) << 4);
+                const bool live = rows[i] != nullptr && bytes != 0;
+                lc_copy16(dst, live ? rows[i] + col : a.wt, live ? bytes : 0u);
+            }
+        };
+        auto split_part = [&](uint32_t big_part, uint32_t small_part) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int row = row0 + 4 * i;
+                const uint32_t off = 128u * row + ((uint32_t)(piece ^ (row & 7)) << 4);
+                lc_split_piece(big_part + off, small_part + off);
+            }
+        };
+        if (a.w_resident) {  // the weight half, once: both parts stay in shared memory for every tile
+            for (int kc = 0; kc < a.k_chunks; ++kc) copy_chunk(w_row, kc, tiles0 + a.w_off + (uint32_t)kc * 2u * kPart);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            for (int kc = 0; kc < a.k_chunks; ++kc) {
+                const uint32_t wb = tiles0 + a.w_off + (uint32_t)kc * 2u * kPart;
+                split_part(wb, wb + kPart);
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            lc_mbar_arrive(w_bar);
+        }
+        const uint32_t lookahead = (uint32_t)a.stages - 1u;  // 1 or 2
+        int s = 0, s_done = 0;
+        uint32_t ph = 0, issued = 0, announced = 0;
+        auto announce = [&]() {  // the oldest unannounced chunk has landed: split it and hand it to the MMA warp
+            const uint32_t base = tiles0 + (uint32_t)s_done * a.stage_stride;
+            split_part(base, base + a.small_off);
+            if (!a.w_resident) split_part(base + kPart, base + a.small_off + kPart);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            lc_mbar_arrive(full_bar(s_done));
+            ++announced;
+            if (++s_done == a.stages) s_done = 0;
+        };
+        bool ok = true;
+        for (int t = first; t < total_tiles && ok; t += step) {
+            const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
+            const float* src_row[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t pos = (int64_t)mt * kLcTileM + row0 + 4 * i;
+                int64_t r = -1;
+                if (pos < a.batch_size) r = a.batch ? (int64_t)__ldg(a.batch + pos) : pos;
+                src_row[i] = (r >= 0 && r < a.n) ? a.hop[hop] + r * a.ldh : nullptr;
+            }
+            for (int kc = 0; kc < a.k_chunks; ++kc) {
+                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error)) {
+                    ok = false;
+                    break;
+                }
+                const uint32_t base = tiles0 + (uint32_t)s * a.stage_stride;
+                copy_chunk(src_row, kc, base);
+                if (!a.w_resident) copy_chunk(w_row, kc, base + kPart);
+                asm volatile("cp.async.commit_group;" ::: "memory");
+                ++issued;
+                if (++s == a.stages) {
+                    s = 0;
+                    ph ^= 1u;
+                }
+                if (issued - announced > lookahead) {
+                    if (lookahead == 1u) {
+                        asm volatile("cp.async.wait_group 1;" ::: "memory");
+                    } else {
+                        asm volatile("cp.async.wait_group 2;" ::: "memory");
+                    }
+                    announce();
+                }
+            }
+        }
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        while (announced < issued) announce();
+    } else if (warp == kLcMmaWarp) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = lc_instr_desc(a.n_half);
+            int s = 0, it = 0;
+            uint32_t ph = 0;
+            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error);
+            for (int t = first; t < total_tiles && ok; t += step, ++it) {
+                const int buf = it & 1;
+                const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+                if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error)) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t tmem_d = tmem_base + (uint32_t)buf * kLcMaxHidden;
+                for (int kc = 0; kc < a.k_chunks; ++kc) {
+                    if (!lc_wait(full_bar(s), ph, abort_flag, a.error)) {
+                        ok = false;
+                        break;
+                    }
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint32_t base = tiles0 + (uint32_t)s * a.stage_stride;
+                    const uint32_t xh = base, xl = base + a.small_off;
+                    const uint32_t wh = a.w_resident ? tiles0 + a.w_off + (uint32_t)kc * 2u * kPart : base + kPart;
+                    const uint32_t wl = a.w_resident ? wh + kPart : base + a.small_off + kPart;
+#pragma unroll
+                    for (int j = 0; j < kLcChunk / 8; ++j) {
+                        const uint32_t o = 32u * j;
+                        // small terms first, the leading term last
+                        lc_mma_tf32(tmem_d, lc_operand_desc(xl + o), lc_operand_desc(wh + o), idesc, (kc | j) != 0);
+                        lc_mma_tf32(tmem_d, lc_operand_desc(xh + o), lc_operand_desc(wl + o), idesc, 1u);
+                        lc_mma_tf32(tmem_d, lc_operand_desc(xh + o), lc_operand_desc(wh + o), idesc, 1u);
+                    }
+                    lc_mma_commit(empty_bar(s));
+                    if (++s == a.stages) {
+                        s = 0;
+                        ph ^= 1u;
+                    }
+                }
+                if (ok) lc_mma_commit(acc_full_bar(buf));
+            }
+            lc_mma_commit(drain_bar);
+            for (uint32_t i = 0; i < kLcSpinLimit; ++i)
+                if (lc_mbar_try_wait(drain_bar, 0)) break;
+        }
+        __syncwarp();
+    } else {
+        lc_epilogue(maps, a, tiles0, tmem_base, acc_full_bar(0), acc_empty_bar(0), abort_flag, first, step, a.n_half,
+                    half * a.n_half);
+    }
+
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == kLcMmaWarp) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kLcTmemCols) : "memory");
+    }
+}
+
 
 int encode_map_2d(const float* base, int64_t inner, int64_t outer, int64_t ld, int box_inner, int box_outer,
                   CUtensorMap* out) {
@@ -469,11 +704,15 @@ using namespace gnnpre;
 
 extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
                                      const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw,
-                                     uint64_t relu_mask, float* Y, int64_t ldy, int64_t y_hop_stride, int32_t* error_flag,
-                                     void* stream) {
+                                     uint64_t relu_mask, int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride,
+                                     int32_t* error_flag, void* stream) {
     if (!hops || num_hops < 1 || num_hops > GNNPRE_MAX_HOPS || !Wt || (!Y && batch_size != 0)) return GNNPRE_ERR_INVALID_ARG;
     if (n < 1 || n > INT32_MAX || feat_dim < 1 || feat_dim > INT32_MAX - kLcChunk || batch_size < 0) return GNNPRE_ERR_INVALID_ARG;
+    if (precision != GNNPRE_LC_TF32 && precision != GNNPRE_LC_TF32X3) return GNNPRE_ERR_INVALID_ARG;
     if (hidden < 16 || hidden > kLcMaxHidden || hidden % 16 != 0) return GNNPRE_ERR_INVALID_ARG;
+    const bool x3 = precision == GNNPRE_LC_TF32X3;
+    const int32_t halves = x3 && hidden > 128 ? 2 : 1;
+    if (halves == 2 && hidden % 64 != 0) return GNNPRE_ERR_INVALID_ARG;  // each half is a whole number of 32-column boxes
     if (ldh < feat_dim || ldw < feat_dim || ldy < hidden) return GNNPRE_ERR_INVALID_ARG;
     if (!batch && batch_size > n) return GNNPRE_ERR_INVALID_ARG;
     if (ldh % 4 != 0 || ldw % 4 != 0 || ldy % 4 != 0 || y_hop_stride % 4 != 0) return GNNPRE_ERR_ALIGN;
@@ -496,15 +735,29 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
     // Shared memory: [operand stages][resident weight, when it fits][8 warps x 1 output box], after the
     // 1024-byte alignment slack.
     const int32_t k_chunks = (int32_t)((feat_dim + kLcChunk - 1) / kLcChunk);
-    const int64_t w_bytes = (int64_t)k_chunks * hidden * 128;
-    const bool resident = w_bytes <= kLcResidentMax;
-    const uint32_t stage_stride = resident ? (uint32_t)kLcABytes : (uint32_t)(kLcABytes + hidden * 128);
-    const int32_t stages =
-        (int32_t)std::min<int64_t>(kLcMaxStages, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
-    const uint32_t w_off = (uint32_t)stages * stage_stride;
+    const int32_t n_half = (int32_t)(hidden / halves);
+    bool resident;
+    uint32_t stage_stride, small_off = 0, w_off;
+    int32_t stages;
+    int64_t w_bytes;
+    if (!x3) {
+        w_bytes = (int64_t)k_chunks * hidden * 128;
+        resident = w_bytes <= kLcResidentMax;
+        stage_stride = resident ? (uint32_t)kLcABytes : (uint32_t)(kLcABytes + hidden * 128);
+        stages = (int32_t)std::min<int64_t>(kLcMaxStages, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
+    } else {
+        // per chunk and operand a high and a low part of 16 KB each (the weight half is padded to 128 rows)
+        w_bytes = (int64_t)k_chunks * 2 * kLcABytes;
+        resident = w_bytes <= kLcResidentMax;
+        small_off = resident ? (uint32_t)kLcABytes : 2u * kLcABytes;
+        stage_stride = 2u * small_off;
+        stages = (int32_t)std::min<int64_t>(3, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
+    }
+    w_off = (uint32_t)stages * stage_stride;
     const uint32_t epi_off = w_off + (resident ? (uint32_t)w_bytes : 0u);
     const size_t smem = 1024 + (size_t)epi_off + 8 * kLcEpiBytes;
-    GNNPRE_CUDA(cudaFuncSetAttribute(k_lc_first_layer, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    auto kernel = x3 ? k_lc_first_layer_x3 : k_lc_first_layer;
+    GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
 
     LcMaps maps;
     GNNPRE_TRY(encode_map_2d(Wt, feat_dim, hidden, ldw, kLcChunk, (int)hidden, &maps.w));
@@ -532,9 +785,14 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
         a.w_resident = resident ? 1 : 0;
         a.w_off = w_off;
         a.epi_off = epi_off;
+        a.wt = Wt;
+        a.ldw = ldw;
+        a.halves = halves;
+        a.n_half = n_half;
+        a.small_off = small_off;
         const int64_t total = (int64_t)kn * tiles_m;
-        const unsigned grid = (unsigned)std::min<int64_t>(num_sms, total);
-        k_lc_first_layer<<<grid, kLcThreads, smem, st>>>(maps, a);
+        const unsigned grid = (unsigned)(std::min<int64_t>(num_sms / halves, total) * halves);
+        kernel<<<grid, kLcThreads, smem, st>>>(maps, a);
         GNNPRE_CUDA(cudaGetLastError());
     }
     return GNNPRE_OK;

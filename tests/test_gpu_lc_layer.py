@@ -7,6 +7,7 @@ Two kinds of comparison:
   * normal inputs: |Y - oracle| <= (2^-9 + F 2^-23) * sum_f |x||w|.  The tensor core reads fp32
     operands as tf32 (relative error below 2^-10 each, so below 2^-9 + 2^-20 per product) and adds in
     fp32 (at most F roundings of 2^-24 each on partial sums bounded by sum |x||w|, doubled for slack).
+    With split operands (GNNPRE_LC_TF32X3) the first term drops to 2^-20.
 """
 import numpy as np
 import pytest
@@ -55,8 +56,12 @@ SHAPES = [
 ]
 
 
+PRECISIONS = (0, 1)  # GNNPRE_LC_TF32, GNNPRE_LC_TF32X3
+
+
+@pytest.mark.parametrize("precision", PRECISIONS)
 @pytest.mark.parametrize("n,F,H,bs,K", SHAPES)
-def test_exact_on_small_integers(B, n, F, H, bs, K):
+def test_exact_on_small_integers(B, n, F, H, bs, K, precision):
     hops_np = [integer_matrix(n, F, 100 + k, -7, 7) for k in range(K)]
     Wt_np = integer_matrix(H, F, 7, -5, 5)
     rng = np.random.default_rng(n + F)
@@ -65,7 +70,7 @@ def test_exact_on_small_integers(B, n, F, H, bs, K):
     Wt = padded_cuda(Wt_np, 5)
     batch = None if bs is None else torch.from_numpy(batch_np.astype(np.int32)).cuda()
     relu_mask = 0b101
-    Y = B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask)
+    Y = B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, precision=precision)
     assert Y.shape == (K, n if bs is None else bs, H)
     for k in range(K):
         want = orc.lc_first_layer(hops_np[k], batch_np, Wt_np, relu=bool((relu_mask >> k) & 1))
@@ -73,8 +78,9 @@ def test_exact_on_small_integers(B, n, F, H, bs, K):
         assert np.array_equal(got, want), f"hop {k}: {np.argwhere(got != want)[:5]}"
 
 
+@pytest.mark.parametrize("precision", PRECISIONS)
 @pytest.mark.parametrize("n,F,H,bs,K", SHAPES[2:7])
-def test_normal_inputs_within_the_tf32_bound(B, n, F, H, bs, K):
+def test_normal_inputs_within_the_bound_of_the_precision(B, n, F, H, bs, K, precision):
     hops_np = [gi.normal_matrix(n, F, 200 + k).numpy() for k in range(K)]
     Wt_np = gi.normal_matrix(H, F, 9).numpy() / np.float32(np.sqrt(F))
     rng = np.random.default_rng(n + H)
@@ -82,12 +88,13 @@ def test_normal_inputs_within_the_tf32_bound(B, n, F, H, bs, K):
     hops = [padded_cuda(h, 2) for h in hops_np]
     Wt = padded_cuda(Wt_np, 1)
     batch = None if bs is None else torch.from_numpy(batch_np.astype(np.int32)).cuda()
-    Y = B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=0b10)
+    Y = B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=0b10, precision=precision)
     for k in range(K):
         relu = k == 1
         want, scale = orc.lc_first_layer(hops_np[k], batch_np, Wt_np, relu=relu, want_abs=True)
         got = to_np(Y[k]).astype(np.float64)
-        bound = (2.0 ** -9 + F * 2.0 ** -23) * scale
+        # split operands: the dropped low x low term and the cut of each low part to tf32 cost 3 * 2^-22 < 2^-20
+        bound = ((2.0 ** -9 if precision == 0 else 2.0 ** -20) + F * 2.0 ** -23) * scale
         assert (np.abs(got - want) <= bound).all(), float((np.abs(got - want) / scale).max())
         # the product is really computed: the error is far below the values themselves
         assert np.abs(got - want).max() < 0.01 * np.abs(want).max()
@@ -155,6 +162,9 @@ def test_bad_arguments_are_refused(B):
         with pytest.raises(B.GnnpreError) as ei:
             B.gnnpre_lc_first_layer([h], None, bad_W)
         assert ei.value.status == -1
+    with pytest.raises(B.GnnpreError) as ei:  # split operands, two column halves: hidden must be a multiple of 64
+        B.gnnpre_lc_first_layer([h], None, torch.zeros((160, 32), device="cuda"), precision=1)
+    assert ei.value.status == -1
     with pytest.raises(B.GnnpreError) as ei:  # leading dimension that is not a multiple of 4
         B.gnnpre_lc_first_layer([torch.zeros((64, 30), device="cuda")], None, torch.zeros((16, 30), device="cuda"))
     assert ei.value.status == -3
@@ -162,3 +172,19 @@ def test_bad_arguments_are_refused(B):
         buf = torch.zeros(64 * 16 + 4, device="cuda")
         B.gnnpre_lc_first_layer([h], None, W, out=buf[1:1 + 64 * 16].view(1, 64, 16))
     assert ei.value.status == -3
+
+
+def test_split_operands_are_far_more_accurate_than_plain_tf32(B):
+    """Same inputs, both precisions: the worst error relative to sum |x||w| falls by more than two orders of
+    magnitude, into the accuracy class of an fp32 dot product of this length (its bound is F 2^-24 = 6e-6)."""
+    n, F, H, bs = 6000, 100, 256, 4096
+    hop_np = gi.normal_matrix(n, F, 31).numpy()
+    Wt_np = gi.normal_matrix(H, F, 32).numpy() / np.float32(np.sqrt(F))
+    batch_np = np.random.default_rng(6).permutation(n)[:bs]
+    want, scale = orc.lc_first_layer(hop_np, batch_np, Wt_np, relu=False, want_abs=True)
+    errs = []
+    for precision in PRECISIONS:
+        Y = B.gnnpre_lc_first_layer([torch.from_numpy(hop_np).cuda()], torch.from_numpy(batch_np.astype(np.int32)).cuda(),
+                                    torch.from_numpy(Wt_np).cuda(), precision=precision)
+        errs.append(float((np.abs(to_np(Y[0]).astype(np.float64) - want) / scale).max()))
+    assert errs[1] < 4e-6 and errs[1] * 100 < errs[0], errs
