@@ -53,6 +53,8 @@ def parse():
                     help="aggregate: the K-hop precomputation (the headline); lc: the first dense stage of an LC model "
                          "(Eq. 9) over the precomputed hops, every row once in a seeded random order")
     ap.add_argument("--hidden", type=int, default=256, help="hidden width of --stage lc")
+    ap.add_argument("--lc-precision", default="tf32", choices=["tf32", "tf32x3"],
+                    help="--stage lc: tf32 operands, or every operand split into two tf32 numbers (fp32-like accuracy)")
     ap.add_argument("--e2e-col-slabs", type=int, default=0, help="column slabs c of the host-buffer run (0 = the library's choice)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -250,19 +252,20 @@ def run_lc_stage(args, w):
     Wt = gi.normal_matrix(H, F, w.seed + 77, device="cuda") / float(np.sqrt(F))
     order = torch.from_numpy(np.random.default_rng(w.seed).permutation(n).astype(np.int32)).cuda()
     relu_mask = (1 << K) - 2  # sigma on every term that has another layer after it (k >= 2 in Eq. 9)
+    prec = B.GNNPRE_LC_TF32X3 if args.lc_precision == "tf32x3" else B.GNNPRE_LC_TF32
     Y = torch.empty((K, n, H), dtype=torch.float32, device="cuda")
-    flag_check = B.gnnpre_lc_first_layer(hops, order[:4096], Wt, relu_mask=relu_mask)  # synchronising call: error word read
+    flag_check = B.gnnpre_lc_first_layer(hops, order[:4096], Wt, relu_mask=relu_mask, precision=prec)  # synchronising call: error word read
     del flag_check
     stream = torch.cuda.current_stream()
 
     def timed(batch, out, steps, warmup):
         for _ in range(warmup):
-            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, out=out, check=False)
+            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, precision=prec, out=out, check=False)
         torch.cuda.synchronize()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
         ev[0].record(stream)
         for i in range(steps):
-            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, out=out, check=False)
+            B.gnnpre_lc_first_layer(hops, batch, Wt, relu_mask=relu_mask, precision=prec, out=out, check=False)
             ev[i + 1].record(stream)
         torch.cuda.synchronize()
         return [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
@@ -284,13 +287,14 @@ def run_lc_stage(args, w):
     line = {
         "metric": "first dense stage of an LC model: output elems/s", "value": elems / (ms_step * 1e-3), "unit": "elems/s",
         "n_gpus": 1, "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
-        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "tf32 inputs, f32 accumulate",
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "tf32 inputs, f32 accumulate" if prec == B.GNNPRE_LC_TF32 else "2 x tf32 per input, f32 accumulate",
         "data": "synthetic", "stage": "lc",
         "config": {"workload": f"{w.name}: first dense stage over the {K} hops of n={n}, F={F}; hidden={H}; all rows, seeded random order",
                    "l2": "inputs and outputs larger than L2", "mini_batch_4096_ms": float(np.median(mini)),
                    "rows_in_order_ms": float(np.median(in_order)), "tflops": 2.0 * K * n * F * H / (ms_step * 1e-3) / 1e12},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": profiled_traffic_lc(K * n) if H == 256 and F == 100 else None, "peak_source": which,
+                     "traffic": profiled_traffic_lc(K * n) if H == 256 and F == 100 and prec == B.GNNPRE_LC_TF32 else None, "peak_source": which,
                      "algorithmic_bytes_per_launch": alg_bytes},
         "gpu_launches": args.steps, "clocks": clocks, "e2e": None,
     }
