@@ -281,8 +281,9 @@ int gnnpre_hop_static(const gnnpre_csr_t* csr, int32_t op, float gin_eps, int64_
  *                     error.  The fastest mode.
  *   GNNPRE_LC_TF32X3  every operand enters as the sum of two tf32 numbers (three tensor-core products per
  *                     term, fp32 accumulation): |error| <= 2^-20 * sum_f |x||w| plus fp32 summation error,
- *                     i.e. fp32-like accuracy.  With hidden > 128 the batch rows are fetched twice and hidden
- *                     must be a multiple of 64 (else INVALID_ARG).
+ *                     i.e. fp32-like accuracy.  A CTA then computes at most 128 output columns: with hidden > 128
+ *                     the batch rows are fetched twice (the second time mostly from L2) and hidden must be a
+ *                     multiple of 64 (else INVALID_ARG).
  * The work is enqueued on `stream` and the call returns without synchronising; nothing is allocated.
  * batch_size = 0 is a no-op.  UNSUPPORTED_ARCH on devices other than compute capability 10.x.
  */

@@ -86,7 +86,7 @@ struct LcArgs {
     // the split-operand kernel only
     const float* wt;       // [hidden, F] weight, leading dimension ldw
     int64_t ldw;
-    int32_t halves;        // CTAs with blockIdx.x % halves == h compute output columns [h n_half, (h + 1) n_half)
+    int32_t halves;        // column parts: CTAs with blockIdx.x % halves == h compute columns [h n_half, (h + 1) n_half)
     int32_t n_half;
     uint32_t small_off;    // offset of the low parts inside a stage
 };
@@ -455,8 +455,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 // that tf32 holds exactly (low 13 mantissa bits cleared) and a low part (the remainder, again cut to
 // what tf32 holds), and  x w  ~=  xh wh + xl wh + xh wl  with fp32 accumulation; the dropped terms are
 // below 2^-21 |x||w|.  Shared memory has to hold both parts of both operands, so a CTA computes at most
-// 128 output columns: with hidden > 128, even and odd CTAs take the two halves and every batch row is
-// gathered by both (the second read mostly hits L2).  No tensor copies on the input side: the producer
+// 128 output columns: with hidden > 128, even and odd CTAs take the two column halves and every batch row is
+// gathered once per part (the later reads mostly hit L2).  No tensor copies on the input side: the producer
 // threads bring rows of the hop matrix AND rows of the weight in with 16-byte asynchronous copies,
 // then read their own pieces back, split them and write the two parts (each thread touches only bytes
 // it copied itself, so the copy's wait_group is all the synchronisation the split needs).
@@ -518,7 +518,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
     const int total_tiles = a.num_hops * a.tiles_m;
     const int half = blockIdx.x % a.halves;
     const int first = blockIdx.x / a.halves, step = gridDim.x / a.halves;
-    constexpr uint32_t kPart = kLcABytes;  // bytes of one [128 rows, 32 floats] part: 16 KB
+    constexpr uint32_t kPart = kLcABytes;               // bytes of one part of the rows' chunk: [128, 32] floats
+    const uint32_t w_part = (uint32_t)a.n_half * 128u;  // bytes of one part of the weight's chunk: [n_half, 32] floats
 
     if (warp < kLcProducerWarps) {
         // ---------------------------------------------------------------- producers
@@ -531,44 +532,47 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
             w_row[i] = r < a.n_half ? a.wt + (int64_t)(half * a.n_half + r) * a.ldw : nullptr;
         }
         // copy this thread's pieces of chunk kc of `rows` (hop rows or weight rows) to `dst_part`
-        auto copy_chunk = [&](const auto& rows, int kc, uint32_t dst_part) {
+        // (a part holds row_limit rows: 128 for the tile, n_half for the weight; rows beyond it do not exist)
+        auto copy_chunk = [&](const auto& rows, int kc, uint32_t dst_part, int row_limit) {
             const int col = kc * kLcChunk + 4 * piece;
             const int left = a.feat_dim - col;
             const uint32_t bytes = left >= 4 ? 16u : left > 0 ? 4u * left : 0u;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int row = row0 + 4 * i;
+                if (row >= row_limit) continue;
                 const uint32_t dst = dst_part + 128u * row + ((uint32_t)(piece ^ (row & 7)) << 4);
                 const bool live = rows[i] != nullptr && bytes != 0;
                 lc_copy16(dst, live ? rows[i] + col : a.wt, live ? bytes : 0u);
             }
         };
-        auto split_part = [&](uint32_t big_part, uint32_t small_part) {
+        auto split_part = [&](uint32_t big_part, uint32_t small_part, int row_limit) {
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const int row = row0 + 4 * i;
+                if (row >= row_limit) continue;
                 const uint32_t off = 128u * row + ((uint32_t)(piece ^ (row & 7)) << 4);
                 lc_split_piece(big_part + off, small_part + off);
             }
         };
         if (a.w_resident) {  // the weight half, once: both parts stay in shared memory for every tile
-            for (int kc = 0; kc < a.k_chunks; ++kc) copy_chunk(w_row, kc, tiles0 + a.w_off + (uint32_t)kc * 2u * kPart);
+            for (int kc = 0; kc < a.k_chunks; ++kc) copy_chunk(w_row, kc, tiles0 + a.w_off + (uint32_t)kc * 2u * w_part, a.n_half);
             asm volatile("cp.async.commit_group;" ::: "memory");
             asm volatile("cp.async.wait_group 0;" ::: "memory");
             for (int kc = 0; kc < a.k_chunks; ++kc) {
-                const uint32_t wb = tiles0 + a.w_off + (uint32_t)kc * 2u * kPart;
-                split_part(wb, wb + kPart);
+                const uint32_t wb = tiles0 + a.w_off + (uint32_t)kc * 2u * w_part;
+                split_part(wb, wb + w_part, a.n_half);
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             lc_mbar_arrive(w_bar);
         }
-        const uint32_t lookahead = (uint32_t)a.stages - 1u;  // 1 or 2
+        const uint32_t lookahead = (uint32_t)a.stages - 1u;  // 1, 2 or 3
         int s = 0, s_done = 0;
         uint32_t ph = 0, issued = 0, announced = 0;
         auto announce = [&]() {  // the oldest unannounced chunk has landed: split it and hand it to the MMA warp
             const uint32_t base = tiles0 + (uint32_t)s_done * a.stage_stride;
-            split_part(base, base + a.small_off);
-            if (!a.w_resident) split_part(base + kPart, base + a.small_off + kPart);
+            split_part(base, base + a.small_off, kLcTileM);
+            if (!a.w_resident) split_part(base + kPart, base + a.small_off + kPart, a.n_half);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             lc_mbar_arrive(full_bar(s_done));
             ++announced;
@@ -591,8 +595,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
                     break;
                 }
                 const uint32_t base = tiles0 + (uint32_t)s * a.stage_stride;
-                copy_chunk(src_row, kc, base);
-                if (!a.w_resident) copy_chunk(w_row, kc, base + kPart);
+                copy_chunk(src_row, kc, base, kLcTileM);
+                if (!a.w_resident) copy_chunk(w_row, kc, base + kPart, a.n_half);
                 asm volatile("cp.async.commit_group;" ::: "memory");
                 ++issued;
                 if (++s == a.stages) {
@@ -602,8 +606,10 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
                 if (issued - announced > lookahead) {
                     if (lookahead == 1u) {
                         asm volatile("cp.async.wait_group 1;" ::: "memory");
-                    } else {
+                    } else if (lookahead == 2u) {
                         asm volatile("cp.async.wait_group 2;" ::: "memory");
+                    } else {
+                        asm volatile("cp.async.wait_group 3;" ::: "memory");
                     }
                     announce();
                 }
@@ -632,8 +638,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint32_t base = tiles0 + (uint32_t)s * a.stage_stride;
                     const uint32_t xh = base, xl = base + a.small_off;
-                    const uint32_t wh = a.w_resident ? tiles0 + a.w_off + (uint32_t)kc * 2u * kPart : base + kPart;
-                    const uint32_t wl = a.w_resident ? wh + kPart : base + a.small_off + kPart;
+                    const uint32_t wh = a.w_resident ? tiles0 + a.w_off + (uint32_t)kc * 2u * w_part : base + kPart;
+                    const uint32_t wl = a.w_resident ? wh + w_part : base + a.small_off + kPart;
 #pragma unroll
                     for (int j = 0; j < kLcChunk / 8; ++j) {
                         const uint32_t o = 32u * j;
@@ -711,8 +717,12 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
     if (precision != GNNPRE_LC_TF32 && precision != GNNPRE_LC_TF32X3) return GNNPRE_ERR_INVALID_ARG;
     if (hidden < 16 || hidden > kLcMaxHidden || hidden % 16 != 0) return GNNPRE_ERR_INVALID_ARG;
     const bool x3 = precision == GNNPRE_LC_TF32X3;
+    // Split operands: both parts of a CTA's weight columns must fit in shared memory, so a CTA computes at most 128
+    // output columns; each part is a whole number of 32-column boxes.  (Parts of 64 columns leave room for four
+    // operand stages instead of two but were measured slower, 8.4 against 4.5 ms on the 2.4 M-row workload: the
+    // per-tile hand-offs, not the stage count, set the pace.)
     const int32_t halves = x3 && hidden > 128 ? 2 : 1;
-    if (halves == 2 && hidden % 64 != 0) return GNNPRE_ERR_INVALID_ARG;  // each half is a whole number of 32-column boxes
+    if (halves == 2 && hidden % 64 != 0) return GNNPRE_ERR_INVALID_ARG;
     if (ldh < feat_dim || ldw < feat_dim || ldy < hidden) return GNNPRE_ERR_INVALID_ARG;
     if (!batch && batch_size > n) return GNNPRE_ERR_INVALID_ARG;
     if (ldh % 4 != 0 || ldw % 4 != 0 || ldy % 4 != 0 || y_hop_stride % 4 != 0) return GNNPRE_ERR_ALIGN;
@@ -746,12 +756,13 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
         stage_stride = resident ? (uint32_t)kLcABytes : (uint32_t)(kLcABytes + hidden * 128);
         stages = (int32_t)std::min<int64_t>(kLcMaxStages, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
     } else {
-        // per chunk and operand a high and a low part of 16 KB each (the weight half is padded to 128 rows)
-        w_bytes = (int64_t)k_chunks * 2 * kLcABytes;
+        // per chunk a high and a low part of the tile's rows (16 KB each) and of the weight part (n_half x 128 B each)
+        const uint32_t w_part = (uint32_t)n_half * 128u;
+        w_bytes = (int64_t)k_chunks * 2 * w_part;
         resident = w_bytes <= kLcResidentMax;
-        small_off = resident ? (uint32_t)kLcABytes : 2u * kLcABytes;
+        small_off = resident ? (uint32_t)kLcABytes : (uint32_t)kLcABytes + w_part;
         stage_stride = 2u * small_off;
-        stages = (int32_t)std::min<int64_t>(3, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
+        stages = (int32_t)std::min<int64_t>(4, (kLcPipeBytes - (resident ? w_bytes : 0)) / stage_stride);
     }
     w_off = (uint32_t)stages * stage_stride;
     const uint32_t epi_off = w_off + (resident ? (uint32_t)w_bytes : 0u);
