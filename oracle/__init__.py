@@ -63,6 +63,7 @@ def _c():
         lib.orc_slab_width.restype = i64
         lib.orc_propagate_blocked.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, ctypes.c_int, i32, i32, p]
         lib.orc_propagate_blocked.restype = ctypes.c_int
+        lib.orc_weighted_hop_sum.argtypes = [ctypes.c_int, f64, i64, p, p, i64, p, i64, ctypes.c_int, p, p]
         lib.orc_lc_first_layer.argtypes = [i64, p, i64, p, i64, i64, p, i64, ctypes.c_int, p, p]
         _lib = lib
     return _lib
@@ -237,3 +238,14 @@ def lc_first_layer(Xk, batch, Wt, relu: bool, want_abs: bool = False):
     _c().orc_lc_first_layer(B, bp, F, _ptr(Xk), ldx, H, _ptr(Wt), ldw, int(bool(relu)), _ptr(Y),
                             _ptr(A) if want_abs else None)
     return (Y, A) if want_abs else Y
+
+
+def weighted_hop_sum(op: int, eps: float, rowptr, colidx, X, gamma) -> np.ndarray:
+    """[n, F] fp64: sum_k gamma[k] A^^k X for k = 0..len(gamma)-1 (fixed-weight generalised PageRank)."""
+    rowptr, colidx, n = _csr(rowptr, colidx)
+    X, ldx = _f32_matrix(X)
+    gamma = np.ascontiguousarray(gamma, dtype=np.float64)
+    Z = np.empty((n, X.shape[1]), dtype=np.float64)
+    _c().orc_weighted_hop_sum(op, float(eps), n, _ptr(rowptr), _ptr(colidx), X.shape[1], _ptr(X), ldx,
+                              gamma.shape[0] - 1, _ptr(gamma), _ptr(Z))
+    return Z

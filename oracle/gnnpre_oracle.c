@@ -25,6 +25,8 @@
  * Parity pins (tests/test_oracle_pins.py): closed forms on complete, cycle, star and regular
  * graphs, fixed points and conservation laws of each operator, brute-force dense A^^k X,
  * an independent scipy.sparse product, and exhaustive checks of the block partition.
+ * The fixed-weight sum of hops, orc_weighted_hop_sum, is pinned by unit weights (one hop each), by the
+ * identity that turns the K-step PageRank iteration into such a sum, and by a closed form on a complete graph.
  * The first dense stage of an LC model (Eq. 9), orc_lc_first_layer, is pinned by a library matrix
  * product, by one-hot / identity weights and by the commutation S^k (X W) = (S^k X) W on integers.
  * Absolute speed is the one thing with no pin: the paper prints ratios only.
@@ -218,6 +220,33 @@ void orc_propagate_teleport(int op, double eps, double alpha, int64_t n, const i
         for (int64_t i = 0; i < n; ++i)
             for (int64_t f = 0; f < F; ++f) xk[i * F + f] = (1.0 - alpha) * xk[i * F + f] + alpha * (double)X[i * ldx + f];
     }
+}
+
+/*
+ * Generalised-PageRank filter with FIXED weights (the appendix on GPRGNN, Eq. 13: H = sum_k gamma_k S^k (...);
+ * with gamma fixed before training it is one more constant filter in the sense of Section 3.1 "Limitation"):
+ *     Z = sum_{k=0..K} gamma[k] A^^k X_0 ,
+ * evaluated hop by hop (A^^k is never formed: same appendix), fp64.  Z is [n, F].
+ */
+void orc_weighted_hop_sum(int op, double eps, int64_t n, const int64_t* rowptr, const int32_t* colidx, int64_t F,
+                          const float* X, int64_t ldx, int K, const double* gamma, double* Z) {
+    const size_t nf = (size_t)n * (size_t)F;
+    double* cur = (double*)malloc(sizeof(double) * nf);
+    double* nxt = (double*)malloc(sizeof(double) * nf);
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t f = 0; f < F; ++f) {
+            cur[i * F + f] = (double)X[i * ldx + f];
+            Z[i * F + f] = gamma[0] * cur[i * F + f];
+        }
+    for (int k = 1; k <= K; ++k) {
+        orc_hop_f64(op, eps, n, rowptr, colidx, F, cur, nxt);
+        for (size_t t = 0; t < nf; ++t) Z[t] += gamma[k] * nxt[t];
+        double* tmp = cur;
+        cur = nxt;
+        nxt = tmp;
+    }
+    free(nxt);
+    free(cur);
 }
 
 /*

@@ -542,3 +542,39 @@ def test_first_layer_commutes_with_propagation():
         hop32 = hops[k].astype(np.float32)
         assert (hop32.astype(np.float64) == hops[k]).all()
         np.testing.assert_array_equal(orc.lc_first_layer(hop32, batch, Wt, relu=False), hops_of_XW[k][batch])
+
+
+# ------------------------------------------------------------------ fixed-weight sum of hops (GPRGNN's filter, weights fixed)
+
+@pytest.mark.parametrize("op", OPS)
+def test_weighted_hop_sum_pins(op):
+    n, F, K = 90, 4, 4
+    rowptr, colidx = random_graph(n, 300, 81)
+    X = features(n, F, 82)
+    hops = orc.propagate(op, EPS, rowptr, colidx, X, K)
+    # unit weights pick single hops (k = 0 is X itself); a general gamma is the same linear combination
+    for k in range(K + 1):
+        e = np.zeros(K + 1)
+        e[k] = 1.0
+        want = X.astype(np.float64) if k == 0 else hops[k - 1]
+        np.testing.assert_allclose(orc.weighted_hop_sum(op, EPS, rowptr, colidx, X, e), want, rtol=1e-13, atol=1e-14)
+    gamma = np.array([0.3, -1.25, 0.5, 2.0, -0.75])
+    want = gamma[0] * X.astype(np.float64) + sum(gamma[k] * hops[k - 1] for k in range(1, K + 1))
+    np.testing.assert_allclose(orc.weighted_hop_sum(op, EPS, rowptr, colidx, X, gamma), want, rtol=1e-12, atol=1e-13)
+    # the K-step PageRank iteration X_k = (1-a) A^ X_{k-1} + a X_0 unrolls to such a sum:
+    # X_K = (1-a)^K A^^K X_0 + a sum_{k<K} (1-a)^k A^^k X_0
+    a = 0.15
+    g = np.array([a * (1 - a) ** k for k in range(K)] + [(1 - a) ** K])
+    ppr = orc.propagate_teleport(op, EPS, a, rowptr, colidx, X, K)[K - 1]
+    np.testing.assert_allclose(orc.weighted_hop_sum(op, EPS, rowptr, colidx, X, g), ppr, rtol=1e-12, atol=1e-13)
+
+
+def test_weighted_hop_sum_on_complete_graph_closed_form():
+    """GCN on K_n: every hop k >= 1 is the column mean, so Z = gamma_0 X + (gamma_1 + ... + gamma_K) mean(X)."""
+    n, F = 7, 3
+    rowptr, colidx = csr_of(n, [(i, j) for i in range(n) for j in range(i + 1, n)])
+    X = features(n, F, 83)
+    gamma = np.array([0.5, 0.25, -2.0, 1.5])
+    mean = X.astype(np.float64).mean(axis=0, keepdims=True)
+    want = gamma[0] * X.astype(np.float64) + gamma[1:].sum() * np.repeat(mean, n, axis=0)
+    np.testing.assert_allclose(orc.weighted_hop_sum(orc.OP_GCN, 0.0, rowptr, colidx, X, gamma), want, rtol=1e-12, atol=1e-13)
