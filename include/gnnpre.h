@@ -252,6 +252,27 @@ int gnnpre_hop_static(const gnnpre_csr_t* csr, int32_t op, float gin_eps, int64_
                       int64_t ldx, float* out, int64_t ldo, void* stream);
 
 /*
+ * K hops as in gnnpre_propagate plus their fixed-weight sum
+ *
+ *     Z = gamma[0] * X_0 + sum_{k=1..K} gamma[k] * X_k ,      X_k = A^ X_{k-1}  (or the plan's teleport recurrence),
+ *
+ * i.e. the generalised-PageRank filter of the appendix on GPRGNN (Eq. 13) with weights fixed before training,
+ * one of the constant filters Section 3.1 "Limitation" allows to precompute.  Z is accumulated in the epilogue
+ * of the kernels that store a finished row, hop by hop (A^^k is never formed), in fp32.
+ *
+ *   plan       a plan whose structure lives on the device; X, out[], Z are DEVICE pointers (no streamed mode)
+ *   gamma      HOST, K + 1 weights
+ *   out        HOST array of K device pointers, as in gnnpre_propagate; when only Z is wanted two buffers can
+ *              alternate (out[k] == out[k-2] is allowed, out[k] == out[k-1] is not: INVALID_ARG)
+ *   Z          device fp32 [n, feat_dim], leading dimension ldz; must not alias X or any out[k]; every element is
+ *              overwritten
+ * Alignment and leading-dimension rules as for gnnpre_propagate (ldz included).  The work is enqueued on `stream`;
+ * the call does not synchronise.
+ */
+int gnnpre_propagate_weighted(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t K, float* const* out, int64_t ldo,
+                              const float* gamma, float* Z, int64_t ldz, void* stream);
+
+/*
  * First dense stage of an LC model on a mini-batch of rows (Eq. 9: every term of COMB begins with the
  * k-th precomputed hop times the first weight matrix; the experimental settings use mini-batches of
  * 4096 rows, hidden width 256 and ReLU).  For each hop matrix k < num_hops:

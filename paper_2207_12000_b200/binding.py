@@ -84,6 +84,8 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
                                      ctypes.POINTER(gnnpre_stats_t)]
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
+    lib.gnnpre_propagate_weighted.argtypes = [p, p, i64, i32, ctypes.POINTER(ctypes.c_void_p), i64,
+                                              ctypes.POINTER(ctypes.c_float), p, i64, p]
     lib.gnnpre_lc_first_layer.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i64, i64, i64, p, i64, p, i64, i64,
                                           ctypes.c_uint64, i32, p, i64, i64, p, p]
     lib.gnnpre_normalize.argtypes = [p, p, i32, p]
@@ -238,6 +240,30 @@ def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: to
     return out
 
 
+def gnnpre_propagate_weighted(plan: Plan, X: torch.Tensor, gamma, *, out=None, Z: torch.Tensor | None = None,
+                              keep_hops: bool = True, stream=None):
+    """K = len(gamma) - 1 hops and Z = gamma[0] X + sum_k gamma[k] X_k, all on the device.
+    Returns (hops, Z); with keep_hops=False two buffers alternate and hops holds only the last two."""
+    K = len(gamma) - 1
+    assert X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    n, F = X.shape
+    Fp = (F + 3) // 4 * 4
+    if out is None:
+        nbuf = K if keep_hops else min(K, 2)
+        bufs = [torch.empty((n, Fp), dtype=torch.float32, device=X.device)[:, :F] for _ in range(nbuf)]
+        out = [bufs[k % nbuf] for k in range(K)]
+    if Z is None:
+        Z = torch.empty((n, Fp), dtype=torch.float32, device=X.device)[:, :F]
+    for o in list(out) + [Z]:
+        assert o.is_cuda and o.dtype == torch.float32 and o.shape == (n, F) and o.stride(1) == 1
+    assert all(o.stride(0) == out[0].stride(0) for o in out)
+    ptrs = (ctypes.c_void_p * K)(*[o.data_ptr() for o in out])
+    g = (ctypes.c_float * (K + 1))(*[float(v) for v in gamma])
+    _check(_lib.gnnpre_propagate_weighted(plan.handle, X.data_ptr(), X.stride(0), K, ptrs, out[0].stride(0), g,
+                                          Z.data_ptr(), Z.stride(0), _stream_ptr(stream)), "gnnpre_propagate_weighted")
+    return list(out), Z
+
+
 GNNPRE_LC_TF32, GNNPRE_LC_TF32X3 = 0, 1
 
 
@@ -321,6 +347,6 @@ def gnnpre_status_string(status: int) -> str:
 
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
-            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_normalize",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_propagate_weighted", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_normalize",
             "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

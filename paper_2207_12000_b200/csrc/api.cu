@@ -64,3 +64,25 @@ extern "C" int gnnpre_propagate(gnnpre_plan_t* P, const float* X, int64_t ldx, i
         return propagate_resident(P, X, ldx, K, out, ldo, st, stats);
     return propagate_streamed(P, X, ldx, x_mem, K, out, ldo, out_mem, st, stats);
 }
+
+extern "C" int gnnpre_propagate_weighted(gnnpre_plan_t* P, const float* X, int64_t ldx, int32_t K, float* const* out,
+                                         int64_t ldo, const float* gamma, float* Z, int64_t ldz, void* stream) {
+    if (!P || !X || !out || !gamma || !Z || K < 1 || K > GNNPRE_MAX_HOPS) return GNNPRE_ERR_INVALID_ARG;
+    if (P->structure_mem != GNNPRE_MEM_DEVICE) return GNNPRE_ERR_INVALID_ARG;  // device-resident plans only
+    if (ldx < P->feat_dim || ldo < P->feat_dim || ldz < P->feat_dim) return GNNPRE_ERR_INVALID_ARG;
+    if (ldx % 4 != 0 || ldo % 4 != 0 || ldz % 4 != 0) return GNNPRE_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(Z) & 15u)) return GNNPRE_ERR_ALIGN;
+    if (Z == X) return GNNPRE_ERR_INVALID_ARG;
+    for (int32_t k = 0; k < K; ++k) {
+        if (!out[k] || out[k] == X || out[k] == Z) return GNNPRE_ERR_INVALID_ARG;
+        if (reinterpret_cast<uintptr_t>(out[k]) & 15u) return GNNPRE_ERR_ALIGN;
+        // a hop may reuse the buffer of the hop before the previous one (two buffers suffice when only Z is wanted),
+        // but never the one it reads
+        if (k > 0 && out[k] == out[k - 1]) return GNNPRE_ERR_INVALID_ARG;
+    }
+    int dev = -1;
+    GNNPRE_CUDA(cudaGetDevice(&dev));
+    if (dev != P->device) return GNNPRE_ERR_INVALID_ARG;
+    WeightedSum w{gamma, Z, ldz};
+    return propagate_resident(P, X, ldx, K, out, ldo, static_cast<cudaStream_t>(stream), nullptr, &w);
+}

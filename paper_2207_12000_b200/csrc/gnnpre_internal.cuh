@@ -176,16 +176,27 @@ struct HopArgs {
     float* xout;             // [n, ldo], likewise
     int64_t ldo;
     int32_t width;           // columns of this slab (multiple of 4)
-    const float* x0;         // [n, ldx0] the slab of X_0, read only when the plan has a teleport term
+    const float* x0;         // [n, ldx0] the slab of X_0, read only when the plan has a teleport term or zsum starts
     int64_t ldx0;
+    // fixed-weight sum of hops, Z = gamma_0 X_0 + sum_k gamma_k X_k (nullptr = none): this hop adds gamma * X_k
+    float* zsum = nullptr;   // [n, ldz], offset to the slab's first column
+    int64_t ldz = 0;
+    float gamma = 0.f;       // weight of the hop being computed
+    float gamma0 = 0.f;      // weight of X_0
+    bool zsum_first = false; // first hop: Z starts from gamma0 * X_0 instead of its old value
 };
 
 // propagate.cu
 int launch_segments(const gnnpre_plan* plan, const HopArgs& a, int64_t seg_lo, int64_t seg_hi, cudaStream_t stream);
 int launch_fixups(const gnnpre_plan* plan, const HopArgs& a, int64_t fix_lo, int64_t fix_hi, cudaStream_t stream);
 int launch_zero_empty_rows(const gnnpre_plan* plan, const HopArgs& a, cudaStream_t stream);
+struct WeightedSum {         // optional extra output of propagate_resident
+    const float* gamma;      // host, K + 1 weights
+    float* Z;                // device [n, ldz]
+    int64_t ldz;
+};
 int propagate_resident(gnnpre_plan* plan, const float* X, int64_t ldx, int32_t K, float* const* out, int64_t ldo,
-                       cudaStream_t stream, gnnpre_stats_t* stats);
+                       cudaStream_t stream, gnnpre_stats_t* stats, const WeightedSum* wsum = nullptr);
 
 // stream.cu
 int propagate_streamed(gnnpre_plan* plan, const float* X, int64_t ldx, int32_t x_mem, int32_t K, float* const* out,

@@ -25,6 +25,11 @@ struct Teleport {
     const float* x0;
     int64_t ldx0;
     float alpha, keep;  // keep = 1 - alpha
+    // fixed-weight sum of hops (zsum == nullptr: none): Z += gamma * (the value stored for this hop)
+    float* zsum;
+    int64_t ldz;
+    float gamma, gamma0;
+    int zsum_first;
 };
 
 __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, const Teleport& tp, int64_t row, int q) {
@@ -35,6 +40,21 @@ __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, cons
         o.y = fmaf(tp.keep, o.y, tp.alpha * z.y);
         o.z = fmaf(tp.keep, o.z, tp.alpha * z.z);
         o.w = fmaf(tp.keep, o.w, tp.alpha * z.w);
+    }
+    if (tp.zsum != nullptr) {  // every finished row piece passes here exactly once per hop
+        float4* zp = reinterpret_cast<float4*>(tp.zsum + row * tp.ldz) + q;
+        float4 acc;
+        if (tp.zsum_first) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(tp.x0 + row * tp.ldx0) + q);
+            acc = make_float4(tp.gamma0 * x.x, tp.gamma0 * x.y, tp.gamma0 * x.z, tp.gamma0 * x.w);
+        } else {
+            acc = *zp;
+        }
+        acc.x = fmaf(tp.gamma, o.x, acc.x);
+        acc.y = fmaf(tp.gamma, o.y, acc.y);
+        acc.z = fmaf(tp.gamma, o.z, acc.z);
+        acc.w = fmaf(tp.gamma, o.w, acc.w);
+        *zp = acc;
     }
     return o;
 }
@@ -420,6 +440,11 @@ Teleport teleport_of(const gnnpre_plan* P, const HopArgs& h, int32_t f0) {
     tp.ldx0 = h.ldx0;
     tp.alpha = h.x0 ? P->teleport_alpha : 0.f;
     tp.keep = (float)(1.0 - (double)tp.alpha);
+    tp.zsum = h.zsum ? h.zsum + f0 : nullptr;
+    tp.ldz = h.ldz;
+    tp.gamma = h.gamma;
+    tp.gamma0 = h.gamma0;
+    tp.zsum_first = h.zsum_first ? 1 : 0;
     return tp;
 }
 
@@ -502,7 +527,7 @@ int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t 
 
 // Everything on the device: K hops, each a sweep over the column slabs and the edge blocks.
 int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, float* const* out, int64_t ldo,
-                       cudaStream_t st, gnnpre_stats_t* stats) {
+                       cudaStream_t st, gnnpre_stats_t* stats, const WeightedSum* wsum) {
     // With stats, events bracket every hop and every launch of the segment kernel.
     std::vector<cudaEvent_t> hop_ev, seg_ev;
     auto mark = [&](std::vector<cudaEvent_t>& v) -> int {
@@ -530,6 +555,13 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
             h.xout = out[k] + f_lo;
             h.ldo = ldo;
             h.width = (int32_t)std::min<int64_t>(P->slab_width, P->feat_dim - f_lo);
+            if (wsum) {
+                h.zsum = wsum->Z + f_lo;
+                h.ldz = wsum->ldz;
+                h.gamma = wsum->gamma[k + 1];
+                h.gamma0 = wsum->gamma[0];
+                h.zsum_first = k == 0;
+            }
             const int tiles = (h.width + kMaxTile - 1) / kMaxTile;
             rc = launch_zero_empty_rows(P, h, st);
             launches += P->num_empty ? 1 : 0;

@@ -417,6 +417,56 @@ def test_teleport_filter_matches_oracle(B, op, alpha):
         B.gnnpre_build_plan(drp, dci, op, 16, teleport_alpha=1.5)
 
 
+@pytest.mark.parametrize("op", OPS)
+def test_weighted_hop_sum_matches_oracle(B, op):
+    """Z = gamma_0 X_0 + sum_k gamma_k X_k accumulated in the kernels' epilogues: every kernel shape, blocks and
+    slabs, a strided Z with untouched padding, hops kept or rotated through two buffers; then on top of the
+    teleport recurrence.  The hops themselves must equal those of gnnpre_propagate bit for bit."""
+    g = gi.rmat(6000, 60000, 33, directed_candidates=True)  # has isolated nodes: SAGE's empty rows are covered
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    gamma = [0.4, -1.5, 0.75, 2.0, -0.6]
+    K = len(gamma) - 1
+    for F, b, c in ((16, 1, 1), (100, 3, 1), (128, 2, 2), (256, 1, 1), (72, 4, 3), (600, 2, 1)):
+        X = gi.normal_matrix(g.n, F, 9, device="cuda")
+        want = orc.weighted_hop_sum(op, EPS, rp, ci, to_np(X), gamma)
+        plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=b, force_col_slabs=c, segment_edges=64)
+        ref, _ = B.gnnpre_propagate(plan, X, K)
+        zbuf = torch.full((g.n, F + 4), -3.0, device="cuda")
+        hops, Z = B.gnnpre_propagate_weighted(plan, X, gamma, Z=zbuf[:, :F])
+        torch.cuda.synchronize()
+        assert hop_error(to_np(Z), want) <= TOL, (F, b, c)
+        assert bool((zbuf[:, F:] == -3.0).all())
+        for k in range(K):
+            assert torch.equal(hops[k], ref[k]), (F, b, c, k)
+        last2, Z2 = B.gnnpre_propagate_weighted(plan, X, gamma, keep_hops=False)
+        torch.cuda.synchronize()
+        assert torch.equal(Z2, Z) and torch.equal(last2[K - 1], ref[K - 1])
+        plan.close()
+    # with a teleport term the summed hops are those of the recurrence
+    F, alpha = 100, 0.2
+    X = gi.normal_matrix(g.n, F, 10, device="cuda")
+    tele = orc.propagate_teleport(op, EPS, alpha, rp, ci, to_np(X), K)
+    want = gamma[0] * to_np(X).astype(np.float64) + sum(gamma[k + 1] * tele[k] for k in range(K))
+    plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=2, teleport_alpha=alpha)
+    _, Z = B.gnnpre_propagate_weighted(plan, X, gamma)
+    torch.cuda.synchronize()
+    assert hop_error(to_np(Z), want) <= TOL
+    # refusals: Z aliasing an input or a hop, a hop written over the one it reads, a plan with host structure
+    with pytest.raises(B.GnnpreError):
+        B.gnnpre_propagate_weighted(plan, X, gamma, Z=X)
+    o = [torch.empty_like(X) for _ in range(2)]
+    with pytest.raises(B.GnnpreError):
+        B.gnnpre_propagate_weighted(plan, X, gamma, out=[o[0], o[0], o[1], o[0]])
+    plan.close()
+    hplan = B.gnnpre_build_plan(g.rowptr.pin_memory(), g.colidx.pin_memory(), op, F, operands_mem=B.GNNPRE_MEM_HOST,
+                                force_blocks=2)
+    if hplan.info()["structure_mem"] == B.GNNPRE_MEM_HOST:
+        with pytest.raises(B.GnnpreError):
+            B.gnnpre_propagate_weighted(hplan, X, gamma)
+    hplan.close()
+
+
 def test_resuming_from_a_finished_hop_gives_the_same_bits(B):
     """Checkpoint/resume: hops 1..2, then hop 3 started from hop 2's output, equal the uninterrupted run."""
     g = gi.rmat(20000, 200000, 29, directed_candidates=True)
