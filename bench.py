@@ -49,6 +49,9 @@ def parse():
     ap.add_argument("--op", type=int, default=-1, help="override the workload's operator (sweeps)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--budget-gb", type=float, default=0.0, help="device-memory budget B_GPU of the streamed plan (0 = free memory)")
+    ap.add_argument("--shard", default="replicas", choices=["replicas", "columns"],
+                    help="N > 1: independent replicas of the workload (weak scaling, the default), or one workload with "
+                         "the feature columns split over the ranks (strong scaling; no collective either)")
     ap.add_argument("--stage", default="aggregate", choices=["aggregate", "lc"],
                     help="aggregate: the K-hop precomputation (the headline); lc: the first dense stage of an LC model "
                          "(Eq. 9) over the precomputed hops, every row once in a seeded random order")
@@ -351,6 +354,14 @@ def main():
     torch.cuda.empty_cache()  # the generator's temporaries go back to the driver: the library allocates with cudaMalloc
     gen_s = time.perf_counter() - t0
     K, F = w.hops, w.feat_dim
+    F_total = F
+    if args.shard == "columns" and world > 1:
+        from paper_2207_12000_b200.shard import column_shard
+        f_lo, f_hi = column_shard(F, world, rank)
+        if f_hi == f_lo:
+            raise SystemExit(f"rank {rank}: more ranks than 4-column slabs of F={F}")
+        X = X[:, f_lo:f_hi]  # a strided view: the library takes the leading dimension
+        F = f_hi - f_lo
     blocks = w.blocks if args.blocks < 0 else args.blocks
     flags = B.GNNPRE_FLAG_LAUNCH_PER_BLOCK if args.per_block_launch else 0
     if args.no_bulk_copy:
@@ -402,8 +413,10 @@ def main():
     step_ms = [a.elapsed_time(b_) for a, b_ in ev]
     total_ms = float(sum(step_ms))
     total_ms = max_over_ranks(total_ms, world, "cuda")
-    units_per_step = K * m * F
-    value = aggregate_throughput(units_per_step, args.steps, world, total_ms)
+    sharded = args.shard == "columns" and world > 1
+    units_per_step = K * m * (F_total if sharded else F)
+    # replicas: every rank does the whole workload; column shards: the ranks share one workload
+    value = aggregate_throughput(units_per_step, args.steps, 1 if sharded else world, total_ms)
 
     # ---------------- roofline of the dominant kernel (the segment kernel: one launch = one hop here)
     peak, peak_kind = measured_peaks()
@@ -448,7 +461,10 @@ def main():
                 _, hst = B.gnnpre_propagate(hplan, Xh, K, outs_h, want_stats=True)
             torch.cuda.synchronize()
             dt = (time.perf_counter() - t0) / reps
-            e2e = {"value": units_per_step / dt, "unit": UNIT, "h2d_bytes_per_step": int(hst.h2d_bytes),
+            # column shards: rank 0 times its own slab through host buffers; the job's figure assumes the other
+            # ranks' slabs (same width but the last) take as long on their own host links
+            e2e_units = K * m * F * world if sharded else units_per_step
+            e2e = {"value": e2e_units / dt, "unit": UNIT, "h2d_bytes_per_step": int(hst.h2d_bytes),
                    "d2h_bytes_per_step": int(hst.d2h_bytes), "ms_per_step": dt * 1e3,
                    "col_slabs": hplan.info()["c"]}
             hinfo = hplan.info()
@@ -490,12 +506,12 @@ def main():
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
-                "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": workload_config(w, g, info), "clocks": clocks.summary(), "e2e": e2e,
+                "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                "config": dict(workload_config(w, g, info), parallelism="column shards" if sharded else "replicas"), "clocks": clocks.summary(), "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "plan_build_ms": plan_ms, "input_generation_s": gen_s,
                 # the same metric if every step also rebuilt the plan (degrees, scales, Eq. 12, edge blocks, segments)
-                "value_including_plan_build": world * units_per_step / ((total_ms / args.steps + plan_ms) * 1e-3),
+                "value_including_plan_build": (1 if sharded else world) * units_per_step / ((total_ms / args.steps + plan_ms) * 1e-3),
                 "hop_ms": [float(st.hop_ms[k]) for k in range(K)]}
         print(json.dumps(line), flush=True)
     plan.close()

@@ -467,6 +467,31 @@ def test_weighted_hop_sum_matches_oracle(B, op):
     hplan.close()
 
 
+@pytest.mark.parametrize("world", [2, 3, 8])
+def test_column_shards_assemble_to_the_full_result(B, world):
+    """Column sharding over `world` ranks, run here one rank after another on the one GPU (the ranks are
+    independent: nothing waits on anything): every rank's slab against the oracle's columns, slabs side by side
+    cover every column once."""
+    from paper_2207_12000_b200.shard import propagate_column_shard
+    g = gi.rmat(8000, 90000, 35, directed_candidates=True)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    F, K, op = 100, 3, 0
+    X = gi.normal_matrix(g.n, F, 3, device="cuda")
+    want = orc.propagate(op, 0.0, rp, ci, to_np(X), K)
+    covered = np.zeros(F, dtype=np.int32)
+    for rank in range(world):
+        lo, outs = propagate_column_shard(B, drp, dci, op, X, K, world, rank)
+        torch.cuda.synchronize()
+        if not outs:
+            continue
+        width = outs[0].shape[1]
+        covered[lo:lo + width] += 1
+        for k in range(K):
+            assert hop_error(to_np(outs[k]), want[k][:, lo:lo + width]) <= TOL, (rank, k)
+    assert (covered == 1).all()
+
+
 def test_resuming_from_a_finished_hop_gives_the_same_bits(B):
     """Checkpoint/resume: hops 1..2, then hop 3 started from hop 2's output, equal the uninterrupted run."""
     g = gi.rmat(20000, 200000, 29, directed_candidates=True)

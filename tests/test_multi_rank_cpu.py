@@ -63,3 +63,51 @@ def test_reference_arm_runs_on_rank0_only():
                         "--gpus", "2", "--steps", "1", "--warmup", "0", "--cpu-seconds", "0.5"], env=env,
                        capture_output=True, text=True, timeout=300)
     assert r.returncode == 0 and '"impl": "reference"' in r.stdout
+
+
+# ------------------------------------------------------------------ column sharding (host logic)
+
+def test_column_shards_tile_the_feature_axis():
+    from paper_2207_12000_b200.shard import column_shard
+    for F in (1, 3, 4, 16, 100, 128, 602, 1433):
+        for world in (1, 2, 3, 4, 8):
+            spans = [column_shard(F, world, r) for r in range(world)]
+            assert spans[0][0] == 0 and spans[-1][1] == F
+            for (a, b), (c, d) in zip(spans, spans[1:]):
+                assert b == c and a <= b and c <= d            # contiguous, in order, possibly empty at the end
+            assert all(lo % 4 == 0 for lo, hi in spans if hi > lo)  # every non-empty slab starts on a 16-byte boundary
+            widths = [hi - lo for lo, hi in spans if hi > lo]
+            w = 4 * -(-F // (4 * world))
+            assert all(x == w for x in widths[:-1]) and 0 < widths[-1] <= w   # equal slabs, a shorter last one
+
+
+def shard_worker(rank, world, port, out):
+    import numpy as np
+    import gnnpre_inputs as gi
+    import oracle as orc
+    from paper_2207_12000_b200.shard import column_shard
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    g = gi.erdos_renyi(300, 1500, 5)
+    X = gi.normal_matrix(300, 22, 6).numpy()
+    K = 2
+    lo, hi = column_shard(X.shape[1], world, rank)
+    # the rank's slab alone (the oracle stands in for the device here: this test is about the partition)
+    mine = orc.propagate(0, 0.0, g.rowptr.numpy(), g.colidx.numpy(), np.ascontiguousarray(X[:, lo:hi]), K)
+    parts = [None] * world
+    dist.all_gather_object(parts, (lo, hi, mine))  # the final placement; nothing crosses ranks before it
+    if rank == 0:
+        full = np.concatenate([p[2] for p in sorted(parts, key=lambda p: p[0])], axis=2)
+        want = orc.propagate(0, 0.0, g.rowptr.numpy(), g.colidx.numpy(), X, K)
+        out["equal"] = bool(np.array_equal(full, want))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_column_sharded_ranks_reproduce_the_unsharded_result():
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    world, port = 2, free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(shard_worker, args=(world, port, out), nprocs=world, join=True)
+        assert out["equal"] is True
