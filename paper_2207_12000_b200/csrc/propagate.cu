@@ -32,6 +32,9 @@ struct Teleport {
     int zsum_first;
 };
 
+// WS: the launch also accumulates the fixed-weight sum of hops.  A compile-time switch, because the mere presence of
+// that code slowed the plain kernels down (L2-resident workloads by 40 %) although its branch was never taken.
+template <bool WS>
 __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, const Teleport& tp, int64_t row, int q) {
     float4 o = make_float4(sum.x * scale, sum.y * scale, sum.z * scale, sum.w * scale);
     if (tp.alpha != 0.f) {
@@ -41,7 +44,7 @@ __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, cons
         o.z = fmaf(tp.keep, o.z, tp.alpha * z.z);
         o.w = fmaf(tp.keep, o.w, tp.alpha * z.w);
     }
-    if (tp.zsum != nullptr) {  // every finished row piece passes here exactly once per hop
+    if (WS) {  // every finished row piece passes here exactly once per hop
         float4* zp = reinterpret_cast<float4*>(tp.zsum + row * tp.ldz) + q;
         float4 acc;
         if (tp.zsum_first) {
@@ -107,7 +110,7 @@ constexpr int kThreads = 256;
 #ifndef GNNPRE_SEG_MIN_BLOCKS
 #define GNNPRE_SEG_MIN_BLOCKS 3
 #endif
-template <int G, int V, int U, int OP, bool HAS_EMPTY>
+template <int G, int V, int U, int OP, bool HAS_EMPTY, bool WS>
 __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -208,7 +211,7 @@ __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(co
                         kahan4(tot[v], cmp[v], acc[v]);
                         if (on[v])
                             reinterpret_cast<float4*>(dst)[gl + v * G] =
-                                partial ? tot[v] : finish_row_piece(tot[v], r, a.tp, row, gl + v * G);
+                                partial ? tot[v] : finish_row_piece<WS>(tot[v], r, a.tp, row, gl + v * G);
                         acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
@@ -268,7 +271,7 @@ struct FixArgs {
 
 // One group per cut row: tail part of its first segment, then the head parts of the following ones,
 // added in segment order.
-template <int G, int V>
+template <int G, int V, bool WS>
 __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -314,39 +317,41 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int q = gl + v * G;
-            if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = finish_row_piece(acc[v], r, a.tp, row, q);
+            if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = finish_row_piece<WS>(acc[v], r, a.tp, row, q);
         }
     }
 }
 
 // Rows without any edge (SAGE, D_i = 0) are zero rows of the result.
 // (With a teleport term they keep alpha * X_0[i].)
+template <bool WS>
 __global__ void k_zero_rows(const int32_t* __restrict__ rows, int64_t count, float* __restrict__ out, int64_t ldo,
                             int32_t f4, const Teleport tp) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count * f4) return;
     const int64_t r = rows[t / f4];
     const int q = (int)(t % f4);
-    *reinterpret_cast<float4*>(out + r * ldo + 4 * q) = finish_row_piece(make_float4(0.f, 0.f, 0.f, 0.f), 0.f, tp, r, q);
+    *reinterpret_cast<float4*>(out + r * ldo + 4 * q) = finish_row_piece<WS>(make_float4(0.f, 0.f, 0.f, 0.f), 0.f, tp, r, q);
 }
 
 template <int G, int V, int U>
 int launch_segments_shape(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int64_t groups = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
+    const bool ws = a.tp.zsum != nullptr;
+#define GNNPRE_LAUNCH_SEGMENTS(OP_, EMPTY_)                                              \
+    do {                                                                                 \
+        if (ws) k_segments<G, V, U, OP_, EMPTY_, true><<<grid, kThreads, 0, st>>>(a);    \
+        else k_segments<G, V, U, OP_, EMPTY_, false><<<grid, kThreads, 0, st>>>(a);      \
+    } while (0)
     switch (P->op) {
-    case GNNPRE_OP_GCN_SYM:
-        k_segments<G, V, U, GNNPRE_OP_GCN_SYM, false><<<grid, kThreads, 0, st>>>(a);
-        break;
-    case GNNPRE_OP_GIN_SUM:
-        k_segments<G, V, U, GNNPRE_OP_GIN_SUM, false><<<grid, kThreads, 0, st>>>(a);
-        break;
+    case GNNPRE_OP_GCN_SYM: GNNPRE_LAUNCH_SEGMENTS(GNNPRE_OP_GCN_SYM, false); break;
+    case GNNPRE_OP_GIN_SUM: GNNPRE_LAUNCH_SEGMENTS(GNNPRE_OP_GIN_SUM, false); break;
     default:
-        if (P->rows_all_nonempty)
-            k_segments<G, V, U, GNNPRE_OP_SAGE_MEAN, false><<<grid, kThreads, 0, st>>>(a);
-        else
-            k_segments<G, V, U, GNNPRE_OP_SAGE_MEAN, true><<<grid, kThreads, 0, st>>>(a);
+        if (P->rows_all_nonempty) GNNPRE_LAUNCH_SEGMENTS(GNNPRE_OP_SAGE_MEAN, false);
+        else GNNPRE_LAUNCH_SEGMENTS(GNNPRE_OP_SAGE_MEAN, true);
     }
+#undef GNNPRE_LAUNCH_SEGMENTS
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }
@@ -390,13 +395,13 @@ int make_row_tensor_map(const float* x, int64_t n, int32_t width, int64_t ldx, C
     return GNNPRE_OK;
 }
 
-template <int OP, bool HAS_EMPTY, int F4C>
+template <int OP, bool HAS_EMPTY, int F4C, bool WS>
 int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int nwarps = tma_warps(a.f4);
     const size_t smem = (size_t)nwarps * kTmaStages * tma_stage_bytes(a.f4);
     CUtensorMap tmap;
     GNNPRE_TRY(make_row_tensor_map(a.x, P->n, 4 * a.f4, a.ldx, &tmap));
-    auto kernel = k_segments_tma<OP, HAS_EMPTY, F4C>;
+    auto kernel = k_segments_tma<OP, HAS_EMPTY, F4C, WS>;
     GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t nseg = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)std::min<int64_t>(P->num_sms, (nseg + nwarps - 1) / nwarps);
@@ -408,9 +413,10 @@ int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream
 // The two widths of the paper's datasets (F = 100, F = 128) get kernels with the row size compiled in.
 template <int OP, bool HAS_EMPTY>
 int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
-    if (a.f4 == 25) return launch_segments_tma_width<OP, HAS_EMPTY, 25>(P, a, st);
-    if (a.f4 == 32) return launch_segments_tma_width<OP, HAS_EMPTY, 32>(P, a, st);
-    return launch_segments_tma_width<OP, HAS_EMPTY, 0>(P, a, st);
+    if (a.tp.zsum != nullptr) return launch_segments_tma_width<OP, HAS_EMPTY, 0, true>(P, a, st);
+    if (a.f4 == 25) return launch_segments_tma_width<OP, HAS_EMPTY, 25, false>(P, a, st);
+    if (a.f4 == 32) return launch_segments_tma_width<OP, HAS_EMPTY, 32, false>(P, a, st);
+    return launch_segments_tma_width<OP, HAS_EMPTY, 0, false>(P, a, st);
 }
 
 int launch_segments_tma(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
@@ -427,7 +433,8 @@ template <int G, int V>
 int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
     const int64_t groups = a.fix_hi - a.fix_lo;
     const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
-    k_row_fixups<G, V><<<grid, kThreads, 0, st>>>(a);
+    if (a.tp.zsum != nullptr) k_row_fixups<G, V, true><<<grid, kThreads, 0, st>>>(a);
+    else k_row_fixups<G, V, false><<<grid, kThreads, 0, st>>>(a);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }
@@ -519,8 +526,10 @@ int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t 
     if (P->num_empty == 0) return GNNPRE_OK;
     const int32_t f4 = h.width / 4;
     const int64_t items = P->num_empty * f4;
-    k_zero_rows<<<(unsigned)((items + 255) / 256), 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4,
-                                                                    teleport_of(P, h, 0));
+    const Teleport tp = teleport_of(P, h, 0);
+    const unsigned grid = (unsigned)((items + 255) / 256);
+    if (tp.zsum != nullptr) k_zero_rows<true><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
+    else k_zero_rows<false><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }

@@ -492,6 +492,41 @@ def test_column_shards_assemble_to_the_full_result(B, world):
     assert (covered == 1).all()
 
 
+def test_propagate_and_first_layer_inside_a_cuda_graph(B):
+    """The device-resident calls only enqueue work, so a CUDA graph can capture them: K hops of configuration 1 and
+    the first dense stage over them, replayed twice on fresh outputs, equal the direct calls bit for bit."""
+    w = gi.WORKLOADS["c1"]
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, w.feat_dim)
+    ref, _ = B.gnnpre_propagate(plan, X, w.hops)
+    Wt = gi.normal_matrix(64, w.feat_dim, 3, device="cuda")
+    batch = torch.arange(0, g.n, 3, dtype=torch.int32, device="cuda")
+    ref_y = B.gnnpre_lc_first_layer(ref, batch, Wt, relu_mask=1)
+    outs = [torch.zeros_like(X) for _ in range(w.hops)]
+    y = torch.zeros_like(ref_y)
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):  # one call outside the capture: one-time set-up of the kernels
+        B.gnnpre_propagate(plan, X, w.hops, outs)
+        B.gnnpre_lc_first_layer(outs, batch, Wt, relu_mask=1, out=y, check=False)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        B.gnnpre_propagate(plan, X, w.hops, outs)
+        B.gnnpre_lc_first_layer(outs, batch, Wt, relu_mask=1, out=y, check=False)
+    for _ in range(2):
+        for o in outs:
+            o.zero_()
+        y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert all(torch.equal(o, r) for o, r in zip(outs, ref)) and torch.equal(y, ref_y)
+    assert int(flag.item()) == 0
+    plan.close()
+
+
 def test_resuming_from_a_finished_hop_gives_the_same_bits(B):
     """Checkpoint/resume: hops 1..2, then hop 3 started from hop 2's output, equal the uninterrupted run."""
     g = gi.rmat(20000, 200000, 29, directed_candidates=True)
