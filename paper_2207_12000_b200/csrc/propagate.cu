@@ -32,19 +32,22 @@ struct Teleport {
     int zsum_first;
 };
 
-// WS: the launch also accumulates the fixed-weight sum of hops.  A compile-time switch, because the mere presence of
-// that code slowed the plain kernels down (L2-resident workloads by 40 %) although its branch was never taken.
-template <bool WS>
+// EP, the epilogue of a finished row: 0 = scale only; 1 = scale and teleport term; 2 = the launch also accumulates the
+// fixed-weight sum of hops (teleport decided at run time).  A compile-time switch, because the mere presence of the
+// optional code slowed the plain kernels down although its branches were never taken (the L2-resident workload by
+// 10 % for the teleport term and by 40 % for the sum).
+constexpr int kEpPlain = 0, kEpTeleport = 1, kEpSum = 2;
+template <int EP>
 __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, const Teleport& tp, int64_t row, int q) {
     float4 o = make_float4(sum.x * scale, sum.y * scale, sum.z * scale, sum.w * scale);
-    if (tp.alpha != 0.f) {
+    if (EP == kEpTeleport || (EP == kEpSum && tp.alpha != 0.f)) {
         const float4 z = __ldg(reinterpret_cast<const float4*>(tp.x0 + row * tp.ldx0) + q);
         o.x = fmaf(tp.keep, o.x, tp.alpha * z.x);
         o.y = fmaf(tp.keep, o.y, tp.alpha * z.y);
         o.z = fmaf(tp.keep, o.z, tp.alpha * z.z);
         o.w = fmaf(tp.keep, o.w, tp.alpha * z.w);
     }
-    if (WS) {  // every finished row piece passes here exactly once per hop
+    if (EP == kEpSum) {  // every finished row piece passes here exactly once per hop
         float4* zp = reinterpret_cast<float4*>(tp.zsum + row * tp.ldz) + q;
         float4 acc;
         if (tp.zsum_first) {
@@ -61,6 +64,9 @@ __device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, cons
     }
     return o;
 }
+
+// Which epilogue a launch needs.
+inline int epilogue_of(const Teleport& tp) { return tp.zsum != nullptr ? kEpSum : tp.alpha != 0.f ? kEpTeleport : kEpPlain; }
 
 struct SegArgs {
     const Segment* segs;
@@ -110,7 +116,7 @@ constexpr int kThreads = 256;
 #ifndef GNNPRE_SEG_MIN_BLOCKS
 #define GNNPRE_SEG_MIN_BLOCKS 3
 #endif
-template <int G, int V, int U, int OP, bool HAS_EMPTY, bool WS>
+template <int G, int V, int U, int OP, bool HAS_EMPTY, int EP>
 __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -211,7 +217,7 @@ __global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(co
                         kahan4(tot[v], cmp[v], acc[v]);
                         if (on[v])
                             reinterpret_cast<float4*>(dst)[gl + v * G] =
-                                partial ? tot[v] : finish_row_piece<WS>(tot[v], r, a.tp, row, gl + v * G);
+                                partial ? tot[v] : finish_row_piece<EP>(tot[v], r, a.tp, row, gl + v * G);
                         acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
                     }
                 }
@@ -271,7 +277,7 @@ struct FixArgs {
 
 // One group per cut row: tail part of its first segment, then the head parts of the following ones,
 // added in segment order.
-template <int G, int V, bool WS>
+template <int G, int V, int EP>
 __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
@@ -317,32 +323,33 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
 #pragma unroll
         for (int v = 0; v < V; ++v) {
             const int q = gl + v * G;
-            if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = finish_row_piece<WS>(acc[v], r, a.tp, row, q);
+            if (q < a.f4) *reinterpret_cast<float4*>(dst + 4 * q) = finish_row_piece<EP>(acc[v], r, a.tp, row, q);
         }
     }
 }
 
 // Rows without any edge (SAGE, D_i = 0) are zero rows of the result.
 // (With a teleport term they keep alpha * X_0[i].)
-template <bool WS>
+template <int EP>
 __global__ void k_zero_rows(const int32_t* __restrict__ rows, int64_t count, float* __restrict__ out, int64_t ldo,
                             int32_t f4, const Teleport tp) {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= count * f4) return;
     const int64_t r = rows[t / f4];
     const int q = (int)(t % f4);
-    *reinterpret_cast<float4*>(out + r * ldo + 4 * q) = finish_row_piece<WS>(make_float4(0.f, 0.f, 0.f, 0.f), 0.f, tp, r, q);
+    *reinterpret_cast<float4*>(out + r * ldo + 4 * q) = finish_row_piece<EP>(make_float4(0.f, 0.f, 0.f, 0.f), 0.f, tp, r, q);
 }
 
 template <int G, int V, int U>
 int launch_segments_shape(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int64_t groups = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
-    const bool ws = a.tp.zsum != nullptr;
-#define GNNPRE_LAUNCH_SEGMENTS(OP_, EMPTY_)                                              \
-    do {                                                                                 \
-        if (ws) k_segments<G, V, U, OP_, EMPTY_, true><<<grid, kThreads, 0, st>>>(a);    \
-        else k_segments<G, V, U, OP_, EMPTY_, false><<<grid, kThreads, 0, st>>>(a);      \
+    const int ep = epilogue_of(a.tp);
+#define GNNPRE_LAUNCH_SEGMENTS(OP_, EMPTY_)                                                                 \
+    do {                                                                                                    \
+        if (ep == kEpSum) k_segments<G, V, U, OP_, EMPTY_, kEpSum><<<grid, kThreads, 0, st>>>(a);           \
+        else if (ep == kEpTeleport) k_segments<G, V, U, OP_, EMPTY_, kEpTeleport><<<grid, kThreads, 0, st>>>(a); \
+        else k_segments<G, V, U, OP_, EMPTY_, kEpPlain><<<grid, kThreads, 0, st>>>(a);                      \
     } while (0)
     switch (P->op) {
     case GNNPRE_OP_GCN_SYM: GNNPRE_LAUNCH_SEGMENTS(GNNPRE_OP_GCN_SYM, false); break;
@@ -395,13 +402,13 @@ int make_row_tensor_map(const float* x, int64_t n, int32_t width, int64_t ldx, C
     return GNNPRE_OK;
 }
 
-template <int OP, bool HAS_EMPTY, int F4C, bool WS>
+template <int OP, bool HAS_EMPTY, int F4C, int EP>
 int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int nwarps = tma_warps(a.f4);
     const size_t smem = (size_t)nwarps * kTmaStages * tma_stage_bytes(a.f4);
     CUtensorMap tmap;
     GNNPRE_TRY(make_row_tensor_map(a.x, P->n, 4 * a.f4, a.ldx, &tmap));
-    auto kernel = k_segments_tma<OP, HAS_EMPTY, F4C, WS>;
+    auto kernel = k_segments_tma<OP, HAS_EMPTY, F4C, EP>;
     GNNPRE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int64_t nseg = a.seg_hi - a.seg_lo;
     const unsigned grid = (unsigned)std::min<int64_t>(P->num_sms, (nseg + nwarps - 1) / nwarps);
@@ -413,10 +420,12 @@ int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream
 // The two widths of the paper's datasets (F = 100, F = 128) get kernels with the row size compiled in.
 template <int OP, bool HAS_EMPTY>
 int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
-    if (a.tp.zsum != nullptr) return launch_segments_tma_width<OP, HAS_EMPTY, 0, true>(P, a, st);
-    if (a.f4 == 25) return launch_segments_tma_width<OP, HAS_EMPTY, 25, false>(P, a, st);
-    if (a.f4 == 32) return launch_segments_tma_width<OP, HAS_EMPTY, 32, false>(P, a, st);
-    return launch_segments_tma_width<OP, HAS_EMPTY, 0, false>(P, a, st);
+    const int ep = epilogue_of(a.tp);
+    if (ep == kEpSum) return launch_segments_tma_width<OP, HAS_EMPTY, 0, kEpSum>(P, a, st);
+    if (ep == kEpTeleport) return launch_segments_tma_width<OP, HAS_EMPTY, 0, kEpTeleport>(P, a, st);
+    if (a.f4 == 25) return launch_segments_tma_width<OP, HAS_EMPTY, 25, kEpPlain>(P, a, st);
+    if (a.f4 == 32) return launch_segments_tma_width<OP, HAS_EMPTY, 32, kEpPlain>(P, a, st);
+    return launch_segments_tma_width<OP, HAS_EMPTY, 0, kEpPlain>(P, a, st);
 }
 
 int launch_segments_tma(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
@@ -433,8 +442,10 @@ template <int G, int V>
 int launch_fixups_shape(const FixArgs& a, cudaStream_t st) {
     const int64_t groups = a.fix_hi - a.fix_lo;
     const unsigned grid = (unsigned)((groups * G + kThreads - 1) / kThreads);
-    if (a.tp.zsum != nullptr) k_row_fixups<G, V, true><<<grid, kThreads, 0, st>>>(a);
-    else k_row_fixups<G, V, false><<<grid, kThreads, 0, st>>>(a);
+    const int ep = epilogue_of(a.tp);
+    if (ep == kEpSum) k_row_fixups<G, V, kEpSum><<<grid, kThreads, 0, st>>>(a);
+    else if (ep == kEpTeleport) k_row_fixups<G, V, kEpTeleport><<<grid, kThreads, 0, st>>>(a);
+    else k_row_fixups<G, V, kEpPlain><<<grid, kThreads, 0, st>>>(a);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }
@@ -528,8 +539,10 @@ int launch_zero_empty_rows(const gnnpre_plan* P, const HopArgs& h, cudaStream_t 
     const int64_t items = P->num_empty * f4;
     const Teleport tp = teleport_of(P, h, 0);
     const unsigned grid = (unsigned)((items + 255) / 256);
-    if (tp.zsum != nullptr) k_zero_rows<true><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
-    else k_zero_rows<false><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
+    const int ep = epilogue_of(tp);
+    if (ep == kEpSum) k_zero_rows<kEpSum><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
+    else if (ep == kEpTeleport) k_zero_rows<kEpTeleport><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
+    else k_zero_rows<kEpPlain><<<grid, 256, 0, st>>>(P->emptyrows.p, P->num_empty, h.xout, h.ldo, f4, tp);
     GNNPRE_CUDA(cudaGetLastError());
     return GNNPRE_OK;
 }

@@ -138,7 +138,7 @@ struct TmaChunk {
 };
 
 // F4C: the row width in float4 when known at compile time (shared-memory offsets become immediates), else 0.
-template <int OP, bool HAS_EMPTY, int F4C, bool WS>
+template <int OP, bool HAS_EMPTY, int F4C, int EP>
 __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
     k_segments_tma(const SegArgs a, const __grid_constant__ CUtensorMap tmap, int* error) {
     constexpr unsigned kFull = 0xffffffffu;
@@ -234,7 +234,7 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
             quad_kahan(tot, cmp, acc);
             if (on) {
                 const float4 sum = make_float4(tot.lo.x, tot.lo.y, tot.hi.x, tot.hi.y);
-                reinterpret_cast<float4*>(dst)[lane] = partial ? sum : finish_row_piece<WS>(sum, r, a.tp, row, lane);
+                reinterpret_cast<float4*>(dst)[lane] = partial ? sum : finish_row_piece<EP>(sum, r, a.tp, row, lane);
             }
             acc = tot = cmp = quad_zero();
         };
