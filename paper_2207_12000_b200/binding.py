@@ -286,6 +286,8 @@ def gnnpre_lc_first_layer(hops, batch, Wt: torch.Tensor, *, relu_mask: int = 0, 
     if batch is None:
         B, bptr = n, None
     else:
+        if batch.dtype == torch.int64:  # the default index type of the host framework; the library takes int32
+            batch = batch.to(torch.int32)
         assert batch.is_cuda and batch.dtype == torch.int32 and batch.dim() == 1 and batch.is_contiguous()
         B, bptr = batch.numel(), batch.data_ptr()
     if out is None:
