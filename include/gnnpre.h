@@ -315,6 +315,19 @@ int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n,
                           uint64_t relu_mask, int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride,
                           int32_t* error_flag, void* stream);
 
+/*
+ * Failure-detection self-test of gnnpre_lc_first_layer's kernel: one launch (one tile of up to 128 rows of `hop`,
+ * tf32 mode) in which the producer warps never announce a chunk, so that every bounded wait of the kernel gives up
+ * after `polls` polls (1..100000; a poll parks the warp for at most 20 us).  The kernel must raise the error word,
+ * let its copies land, free its tensor memory and return; the call synchronises the stream and returns
+ * GNNPRE_ERR_TIMEOUT when the error word was raised (the expected outcome), GNNPRE_OK otherwise.  No wait is
+ * unbounded and nothing faults: the device stays usable and a following gnnpre_lc_first_layer call must succeed.
+ * Arguments as for gnnpre_lc_first_layer (device pointers; error_flag required; Y receives nothing meaningful).
+ */
+int gnnpre_lc_selftest_wait_timeout(const float* hop, int64_t n, int64_t feat_dim, int64_t ldh, const float* Wt,
+                                    int64_t hidden, int64_t ldw, float* Y, int64_t ldy, int32_t* error_flag,
+                                    uint32_t polls, void* stream);
+
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;
  * ties towards smaller c, then smaller b.  BUDGET_TOO_SMALL if infeasible.  Host only. */

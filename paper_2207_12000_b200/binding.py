@@ -84,6 +84,7 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_propagate.argtypes = [p, p, i64, i32, i32, ctypes.POINTER(p), i64, i32, p,
                                      ctypes.POINTER(gnnpre_stats_t)]
     lib.gnnpre_hop_static.argtypes = [ctypes.POINTER(gnnpre_csr_t), i32, ctypes.c_float, i64, p, i64, p, i64, p]
+    lib.gnnpre_lc_selftest_wait_timeout.argtypes = [p, i64, i64, i64, p, i64, i64, p, i64, p, ctypes.c_uint32, p]
     lib.gnnpre_propagate_weighted.argtypes = [p, p, i64, i32, ctypes.POINTER(ctypes.c_void_p), i64,
                                               ctypes.POINTER(ctypes.c_float), p, i64, p]
     lib.gnnpre_lc_first_layer.argtypes = [ctypes.POINTER(ctypes.c_void_p), i32, i64, i64, i64, p, i64, p, i64, i64,
@@ -240,6 +241,16 @@ def gnnpre_hop_static(rowptr: torch.Tensor, colidx: torch.Tensor, op: int, X: to
     return out
 
 
+def gnnpre_lc_selftest_wait_timeout(hop: torch.Tensor, Wt: torch.Tensor, polls: int = 200, stream=None) -> int:
+    """Status of a first-layer launch whose waits are made to run out (expected: -8, GNNPRE_ERR_TIMEOUT)."""
+    n, F = hop.shape
+    H = Wt.shape[0]
+    Y = torch.empty((min(n, 128), H), dtype=torch.float32, device=hop.device)
+    flag = torch.zeros(1, dtype=torch.int32, device=hop.device)
+    return int(_lib.gnnpre_lc_selftest_wait_timeout(hop.data_ptr(), n, F, hop.stride(0), Wt.data_ptr(), H, Wt.stride(0),
+                                                    Y.data_ptr(), Y.stride(0), flag.data_ptr(), polls, _stream_ptr(stream)))
+
+
 def gnnpre_propagate_weighted(plan: Plan, X: torch.Tensor, gamma, *, out=None, Z: torch.Tensor | None = None,
                               keep_hops: bool = True, stream=None):
     """K = len(gamma) - 1 hops and Z = gamma[0] X + sum_k gamma[k] X_k, all on the device.
@@ -349,6 +360,6 @@ def gnnpre_status_string(status: int) -> str:
 
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
-            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_propagate_weighted", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_normalize",
+            "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_propagate_weighted", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_lc_selftest_wait_timeout", "gnnpre_normalize",
             "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

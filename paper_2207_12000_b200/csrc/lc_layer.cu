@@ -89,6 +89,9 @@ struct LcArgs {
     int32_t halves;        // column parts: CTAs with blockIdx.x % halves == h compute columns [h n_half, (h + 1) n_half)
     int32_t n_half;
     uint32_t small_off;    // offset of the low parts inside a stage
+    // failure-detection self-test: the producers never announce a chunk, so every wait runs out
+    int32_t drop_announcements;
+    uint32_t spin_limit;   // polls before a wait gives up
 };
 
 __device__ __forceinline__ uint32_t lc_smem_u32(const void* p) {
@@ -121,8 +124,9 @@ __device__ __forceinline__ bool lc_mbar_try_wait(uint32_t bar, uint32_t parity) 
 
 // Bounded wait.  False when the limit ran out (the abort flag and the error word are then set) or
 // when another role has already given up.
-__device__ __forceinline__ bool lc_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* error) {
-    for (uint32_t i = 0; i < kLcSpinLimit; ++i) {
+__device__ __forceinline__ bool lc_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int32_t* error,
+                                        uint32_t limit = kLcSpinLimit) {
+    for (uint32_t i = 0; i < limit; ++i) {
         if (lc_mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
     }
@@ -217,7 +221,7 @@ __device__ __forceinline__ void lc_epilogue(const LcMaps& maps, const LcArgs& a,
         const int hop = t / a.tiles_m, mt = t - hop * a.tiles_m;
         const int buf = it & 1;
         const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-        if (!__all_sync(0xffffffffu, lc_wait(acc_full0 + 8u * buf, acc_ph, abort_flag, a.error))) break;
+        if (!__all_sync(0xffffffffu, lc_wait(acc_full0 + 8u * buf, acc_ph, abort_flag, a.error, a.spin_limit))) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const bool relu = (a.relu_mask >> hop) & 1u;
         const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)buf * kLcMaxHidden;
@@ -337,7 +341,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
                 src_row[i] = (r >= 0 && r < a.n) ? a.hop[hop] + r * a.ldh : nullptr;
             }
             for (int kc = 0; kc < a.k_chunks; ++kc) {
-                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error)) {
+                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error, a.spin_limit)) {
                     ok = false;
                     break;
                 }
@@ -367,7 +371,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
                     // all but the newest kLcLookahead groups have landed: hand the oldest to the MMA warp
                     asm volatile("cp.async.wait_group %0;" ::"n"(kLcLookahead) : "memory");
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    lc_mbar_arrive(full_bar(s_done));
+                    if (!a.drop_announcements) lc_mbar_arrive(full_bar(s_done));
                     ++announced;
                     if (++s_done == a.stages) s_done = 0;
                 }
@@ -377,7 +381,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         while (announced < issued) {
-            lc_mbar_arrive(full_bar(s_done));
+            if (!a.drop_announcements) lc_mbar_arrive(full_bar(s_done));
             ++announced;
             if (++s_done == a.stages) s_done = 0;
         }
@@ -403,15 +407,15 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
             const uint32_t idesc = lc_instr_desc(a.hidden);
             int s = 0, it = 0;
             uint32_t ph = 0;
-            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error);
+            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error, a.spin_limit);
             for (int t = blockIdx.x; t < total_tiles && ok; t += gridDim.x, ++it) {
                 const int buf = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-                if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error)) break;
+                if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error, a.spin_limit)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + (uint32_t)buf * kLcMaxHidden;
                 for (int kc = 0; kc < a.k_chunks; ++kc) {
-                    if (!lc_wait(full_bar(s), ph, abort_flag, a.error)) {
+                    if (!lc_wait(full_bar(s), ph, abort_flag, a.error, a.spin_limit)) {
                         ok = false;
                         break;
                     }
@@ -590,7 +594,7 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
                 src_row[i] = (r >= 0 && r < a.n) ? a.hop[hop] + r * a.ldh : nullptr;
             }
             for (int kc = 0; kc < a.k_chunks; ++kc) {
-                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error)) {
+                if (!lc_wait(empty_bar(s), ph ^ 1u, abort_flag, a.error, a.spin_limit)) {
                     ok = false;
                     break;
                 }
@@ -623,15 +627,15 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer_x3(const __gri
             const uint32_t idesc = lc_instr_desc(a.n_half);
             int s = 0, it = 0;
             uint32_t ph = 0;
-            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error);
+            bool ok = !a.w_resident || lc_wait(w_bar, 0, abort_flag, a.error, a.spin_limit);
             for (int t = first; t < total_tiles && ok; t += step, ++it) {
                 const int buf = it & 1;
                 const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-                if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error)) break;
+                if (!lc_wait(acc_empty_bar(buf), acc_ph ^ 1u, abort_flag, a.error, a.spin_limit)) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint32_t tmem_d = tmem_base + (uint32_t)buf * kLcMaxHidden;
                 for (int kc = 0; kc < a.k_chunks; ++kc) {
-                    if (!lc_wait(full_bar(s), ph, abort_flag, a.error)) {
+                    if (!lc_wait(full_bar(s), ph, abort_flag, a.error, a.spin_limit)) {
                         ok = false;
                         break;
                     }
@@ -708,10 +712,11 @@ int encode_map_2d(const float* base, int64_t inner, int64_t outer, int64_t ld, i
 
 using namespace gnnpre;
 
-extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
-                                     const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw,
-                                     uint64_t relu_mask, int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride,
-                                     int32_t* error_flag, void* stream) {
+// selftest_polls > 0: the producers announce nothing and every wait gives up after that many polls.
+static int lc_launch(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
+                     const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw, uint64_t relu_mask,
+                     int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride, int32_t* error_flag, void* stream,
+                     uint32_t selftest_polls) {
     if (!hops || num_hops < 1 || num_hops > GNNPRE_MAX_HOPS || !Wt || (!Y && batch_size != 0)) return GNNPRE_ERR_INVALID_ARG;
     if (n < 1 || n > INT32_MAX || feat_dim < 1 || feat_dim > INT32_MAX - kLcChunk || batch_size < 0) return GNNPRE_ERR_INVALID_ARG;
     if (precision != GNNPRE_LC_TF32 && precision != GNNPRE_LC_TF32X3) return GNNPRE_ERR_INVALID_ARG;
@@ -801,10 +806,37 @@ extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops,
         a.halves = halves;
         a.n_half = n_half;
         a.small_off = small_off;
+        a.drop_announcements = selftest_polls > 0 ? 1 : 0;
+        a.spin_limit = selftest_polls > 0 ? selftest_polls : kLcSpinLimit;
         const int64_t total = (int64_t)kn * tiles_m;
         const unsigned grid = (unsigned)(std::min<int64_t>(num_sms / halves, total) * halves);
         kernel<<<grid, kLcThreads, smem, st>>>(maps, a);
         GNNPRE_CUDA(cudaGetLastError());
     }
     return GNNPRE_OK;
+}
+
+extern "C" int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n, int64_t feat_dim, int64_t ldh,
+                                     const int32_t* batch, int64_t batch_size, const float* Wt, int64_t hidden, int64_t ldw,
+                                     uint64_t relu_mask, int32_t precision, float* Y, int64_t ldy, int64_t y_hop_stride,
+                                     int32_t* error_flag, void* stream) {
+    return lc_launch(hops, num_hops, n, feat_dim, ldh, batch, batch_size, Wt, hidden, ldw, relu_mask, precision, Y, ldy,
+                     y_hop_stride, error_flag, stream, 0);
+}
+
+// Failure-detection self-test: see include/gnnpre.h.
+extern "C" int gnnpre_lc_selftest_wait_timeout(const float* hop, int64_t n, int64_t feat_dim, int64_t ldh, const float* Wt,
+                                               int64_t hidden, int64_t ldw, float* Y, int64_t ldy, int32_t* error_flag,
+                                               uint32_t polls, void* stream) {
+    if (!error_flag || polls == 0 || polls > 100000u) return GNNPRE_ERR_INVALID_ARG;
+    const float* hops[1] = {hop};
+    const int64_t rows = n < kLcTileM ? n : kLcTileM;  // one tile, one CTA
+    GNNPRE_CUDA(cudaMemsetAsync(error_flag, 0, sizeof(int32_t), static_cast<cudaStream_t>(stream)));
+    const int rc = lc_launch(hops, 1, n, feat_dim, ldh, nullptr, rows, Wt, hidden, ldw, 0, GNNPRE_LC_TF32, Y, ldy, 0, error_flag,
+                             stream, polls);
+    if (rc != GNNPRE_OK) return rc;
+    GNNPRE_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    int32_t flag = 0;
+    GNNPRE_CUDA(cudaMemcpy(&flag, error_flag, sizeof(flag), cudaMemcpyDeviceToHost));
+    return flag ? GNNPRE_ERR_TIMEOUT : GNNPRE_OK;
 }

@@ -188,3 +188,16 @@ def test_split_operands_are_far_more_accurate_than_plain_tf32(B):
                                     torch.from_numpy(Wt_np).cuda(), precision=precision)
         errs.append(float((np.abs(to_np(Y[0]).astype(np.float64) - want) / scale).max()))
     assert errs[1] < 4e-6 and errs[1] * 100 < errs[0], errs
+
+
+def test_waits_that_run_out_are_reported_and_the_device_stays_usable(B):
+    """Failure detection without a fault: the producers announce nothing, every bounded wait of the kernel gives
+    up, the call reports TIMEOUT (-8); tensor memory was freed, so the next call runs and is exact."""
+    n, F, H = 500, 100, 256
+    hop_np = integer_matrix(n, F, 1, -4, 4)
+    Wt_np = integer_matrix(H, F, 2, -4, 4)
+    hop, Wt = torch.from_numpy(hop_np).cuda(), torch.from_numpy(Wt_np).cuda()
+    for _ in range(2):
+        assert B.gnnpre_lc_selftest_wait_timeout(hop, Wt, polls=200) == -8
+        Y = B.gnnpre_lc_first_layer([hop], None, Wt)
+        assert np.array_equal(to_np(Y[0]).astype(np.float64), orc.lc_first_layer(hop_np, None, Wt_np, relu=False))
