@@ -16,9 +16,10 @@
 //            operands read from shared memory through swizzled K-major descriptors, fp32 accumulator
 //            in tensor memory) and hands stages back with tcgen05.commit on the `empty` mbarrier.
 //   warps 5-12  epilogue.  Two warps share each quarter of the accumulator's 128 lanes (even and odd
-//            column boxes); a warp pulls its part out of tensor memory with tcgen05.ld 32 columns at a time, applies ReLU where asked, lays the
-//            [32, 32] box down in shared memory (128-byte swizzle, conflict-free) and hands it to the
-//            copy engine as a tensor store, which writes whole lines and clips the ragged edges.
+//            column boxes); a warp pulls its part out of tensor memory with tcgen05.ld 32 columns at a
+//            time, applies ReLU where asked, lays the [32, 32] box down in shared memory (128-byte
+//            swizzle, conflict-free) and hands it to the copy engine as a tensor store, which writes
+//            whole lines and clips the ragged edges.
 //
 // A weight of up to 128 KB is loaded once per CTA and stays in shared memory; a larger one is
 // streamed chunk by chunk beside the rows.
@@ -26,8 +27,9 @@
 // one tile overlaps the copies and MMAs of the next.  The gathered rows never exist in HBM as a
 // matrix of their own: the gather is the A-operand load.
 //
-// Arithmetic: the tensor core reads the fp32 operands as tf32 (it ignores the low 13 mantissa bits)
-// and accumulates in fp32.
+// Arithmetic: the tensor core reads the fp32 operands as tf32 (8 exponent bits, 10 explicit mantissa
+// bits: a relative error below 2^-10 per operand) and accumulates in fp32.  k_lc_first_layer_x3 below
+// feeds every operand as two tf32 numbers instead.
 //
 // Every wait is bounded.  A wait that runs out raises the CTA's abort flag and the caller's error
 // word; every role then leaves its loop, the producers wait for the copies they still have in
