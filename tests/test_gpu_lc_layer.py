@@ -51,6 +51,8 @@ SHAPES = [
     (777, 13, 48, 300, 2),      # fewer features than one chunk
     (2000, 602, 64, 517, 1),    # Reddit's width: 19 chunks, pad columns full of NaN
     (517, 40, 80, None, 2),     # no batch: every row
+    (1500, 200, 256, 700, 2),   # a weight too large to stay in shared memory at full hidden width: streamed beside the rows
+    (900, 300, 192, 333, 1),    # hidden = 192: two column halves of 96 in the split-operand mode
     (400, 8, 16, 1, 1),         # a single row
     (50000, 100, 256, 50000, 3),  # more tiles than SMs: persistent loop, both accumulator buffers, many phases
 ]
@@ -79,7 +81,7 @@ def test_exact_on_small_integers(B, n, F, H, bs, K, precision):
 
 
 @pytest.mark.parametrize("precision", PRECISIONS)
-@pytest.mark.parametrize("n,F,H,bs,K", SHAPES[2:7])
+@pytest.mark.parametrize("n,F,H,bs,K", SHAPES[2:9])
 def test_normal_inputs_within_the_bound_of_the_precision(B, n, F, H, bs, K, precision):
     hops_np = [gi.normal_matrix(n, F, 200 + k).numpy() for k in range(K)]
     Wt_np = gi.normal_matrix(H, F, 9).numpy() / np.float32(np.sqrt(F))
