@@ -297,8 +297,8 @@ int gnnpre_propagate_weighted(gnnpre_plan_t* plan, const float* X, int64_t ldx, 
  * ldh, ldw >= feat_dim and ldy >= hidden (else INVALID_ARG); ldh, ldw, ldy, y_hop_stride multiples of 4
  * and all base pointers 16-byte aligned (else ALIGN).  feat_dim itself may be any value >= 1.
  * Arithmetic, by `precision`:
- *   GNNPRE_LC_TF32    tensor cores with tf32 inputs (the fp32 operands are read with 10 explicit mantissa
- *                     bits) and fp32 accumulation: |error| <= 2^-9 * sum_f |x||w| plus fp32 summation
+ *   GNNPRE_LC_TF32    tensor cores with tf32 inputs (the low 13 mantissa bits of the fp32 operands are cut,
+ *                     not rounded) and fp32 accumulation: |error| <= 2^-9 * sum_f |x||w| plus fp32 summation
  *                     error.  The fastest mode.
  *   GNNPRE_LC_TF32X3  every operand enters as the sum of two tf32 numbers (three tensor-core products per
  *                     term, fp32 accumulation): |error| <= 2^-20 * sum_f |x||w| plus fp32 summation error,

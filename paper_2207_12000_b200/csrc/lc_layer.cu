@@ -28,7 +28,7 @@
 // matrix of their own: the gather is the A-operand load.
 //
 // Arithmetic: the tensor core reads the fp32 operands as tf32 (8 exponent bits, 10 explicit mantissa
-// bits: a relative error below 2^-10 per operand) and accumulates in fp32.  k_lc_first_layer_x3 below
+// bits; the low 13 bits are cut, not rounded: a relative error below 2^-10 per operand) and accumulates in fp32.  k_lc_first_layer_x3 below
 // feeds every operand as two tf32 numbers instead.
 //
 // Every wait is bounded.  A wait that runs out raises the CTA's abort flag and the caller's error
@@ -458,8 +458,8 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 
 // ------------------------------------------------------------------------------------------------
 // The same stage with fp32-like accuracy ("3 x tf32"): every fp32 operand is split into a high part
-// that tf32 holds exactly (low 13 mantissa bits cleared) and a low part (the remainder, again cut to
-// what tf32 holds), and  x w  ~=  xh wh + xl wh + xh wl  with fp32 accumulation; the dropped terms are
+// that tf32 holds exactly (low 13 mantissa bits cleared) and a low part (the exact remainder, which the
+// tensor core again reads as tf32), and  x w  ~=  xh wh + xl wh + xh wl  with fp32 accumulation; the dropped terms are
 // below 2^-21 |x||w|.  Shared memory has to hold both parts of both operands, so a CTA computes at most
 // 128 output columns: with hidden > 128, even and odd CTAs take the two column halves and every batch row is
 // gathered once per part (the later reads mostly hit L2).  No tensor copies on the input side: the producer
@@ -467,15 +467,17 @@ __global__ void __launch_bounds__(kLcThreads, 1) k_lc_first_layer(const __grid_c
 // then read their own pieces back, split them and write the two parts (each thread touches only bytes
 // it copied itself, so the copy's wait_group is all the synchronisation the split needs).
 __device__ __forceinline__ void lc_split_piece(uint32_t big_addr, uint32_t small_addr) {
+    // The tensor core ignores the low 13 mantissa bits of an fp32 operand (checked on the device: 1 + 7 * 2^-13
+    // enters a product as 1), so the tile as it was copied already acts as the high part; only the low part
+    // is computed and stored.
     uint32_t v[4];
     asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]) : "r"(big_addr) : "memory");
-    uint32_t hi[4], lo[4];
+    uint32_t lo[4];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        hi[j] = v[j] & 0xffffe000u;
-        lo[j] = __float_as_uint(__uint_as_float(v[j]) - __uint_as_float(hi[j])) & 0xffffe000u;  // the difference is exact
+        const uint32_t hi = v[j] & 0xffffe000u;
+        lo[j] = __float_as_uint(__uint_as_float(v[j]) - __uint_as_float(hi));  // exact; read by the tensor core as tf32
     }
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(big_addr), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]), "r"(hi[3]) : "memory");
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(small_addr), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]), "r"(lo[3]) : "memory");
 }
 
