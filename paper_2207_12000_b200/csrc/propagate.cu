@@ -293,29 +293,48 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
     float4 acc[V], cmp[V];
 #pragma unroll
     for (int v = 0; v < V; ++v) acc[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+    // A hub row spans hundreds of segments and its parts must be added in segment order, so the chain is bound by
+    // load latency: the slot numbers of the next G segments are fetched while the current ones are added, and the
+    // parts themselves are loaded kBatch at a time before they join the sum (the order of the additions is unchanged).
+    constexpr int kBatch = V == 1 ? 8 : V == 2 ? 4 : 2;
+    auto slot_of = [&](int s0_) {
+        int slot = -1;
+        const int s = s0_ + gl;
+        if (s <= last) slot = s == first ? a.segs[s].slot_tail : a.segs[s].slot_head;
+        return slot;
+    };
     int s0 = first;
+    int slot = slot_of(s0);
     while (__any_sync(kFull, s0 <= last)) {
         const int cnt = last - s0 + 1 >= G ? G : (last >= s0 ? last - s0 + 1 : 0);
-        int slot = -1;
-        if (gl < cnt) {
-            const int s = s0 + gl;
-            slot = s == first ? a.segs[s].slot_tail : a.segs[s].slot_head;
-        }
+        const int slot_next = slot_of(s0 + G);
         const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
-        for (int t = 0; t < cnt_max; ++t) {
-            const int sl = __shfl_sync(kFull, slot, t, G);
-            if (t < cnt && sl >= 0) {
-                const float* p = a.scratch + (int64_t)sl * a.scratch_ld;
+        for (int t0 = 0; t0 < cnt_max; t0 += kBatch) {
+            float4 part[kBatch][V];
+            bool live[kBatch];
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                const int t = t0 + u;
+                const int sl = __shfl_sync(kFull, slot, t & (G - 1), G);
+                live[u] = t < cnt && sl >= 0;
+                const float* p = a.scratch + (int64_t)(live[u] ? sl : 0) * a.scratch_ld;
 #pragma unroll
                 for (int v = 0; v < V; ++v) {
                     const int q = gl + v * G;
-                    if (q < a.f4) {
-                        kahan4(acc[v], cmp[v], *reinterpret_cast<const float4*>(p + 4 * q));
-                    }
+                    part[u][v] = live[u] && q < a.f4 ? *reinterpret_cast<const float4*>(p + 4 * q) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kBatch; ++u) {
+                if (live[u]) {
+#pragma unroll
+                    for (int v = 0; v < V; ++v)
+                        if (gl + v * G < a.f4) kahan4(acc[v], cmp[v], part[u][v]);
                 }
             }
         }
         s0 += G;
+        slot = slot_next;
     }
     if (i < a.fix_hi) {
         const float r = a.rscale[row];
