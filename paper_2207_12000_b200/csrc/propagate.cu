@@ -296,7 +296,7 @@ __global__ void __launch_bounds__(kThreads) k_row_fixups(const FixArgs a) {
     // A hub row spans hundreds of segments and its parts must be added in segment order, so the chain is bound by
     // load latency: the slot numbers of the next G segments are fetched while the current ones are added, and the
     // parts themselves are loaded kBatch at a time before they join the sum (the order of the additions is unchanged).
-    constexpr int kBatch = V == 1 ? 8 : V == 2 ? 4 : 2;
+    constexpr int kBatch = 16 / V;  // 64 registers of parts in flight per lane
     auto slot_of = [&](int s0_) {
         int slot = -1;
         const int s = s0_ + gl;
