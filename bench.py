@@ -47,6 +47,8 @@ def parse():
     ap.add_argument("--no-bulk-copy", action="store_true", help="register-gather kernel for every width")
     ap.add_argument("--feat-dim", type=int, default=0, help="override the workload's F (sweeps)")
     ap.add_argument("--op", type=int, default=-1, help="override the workload's operator (sweeps)")
+    ap.add_argument("--ld", type=int, default=0, help="leading dimension (floats) of X and of every hop, e.g. 128 for "
+                                                      "F=100 so that rows start on 512-byte boundaries (0 = F)")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
     ap.add_argument("--budget-gb", type=float, default=0.0, help="device-memory budget B_GPU of the streamed plan (0 = free memory)")
     ap.add_argument("--shard", default="replicas", choices=["replicas", "columns"],
@@ -377,7 +379,14 @@ def main():
     plan_ms = (time.perf_counter() - t0) * 1e3
     info = plan.info()
     m = info["nnz_tilde"]
-    outs = [torch.empty((g.n, F), dtype=torch.float32, device="cuda") for _ in range(K)]
+    if args.ld:  # rows padded to the given leading dimension: strided views, the library takes ldx / ldo
+        assert args.ld >= F and args.ld % 4 == 0 and not (args.shard == "columns" and world > 1)
+        Xp = torch.zeros((g.n, args.ld), dtype=torch.float32, device="cuda")
+        Xp[:, :F] = X
+        X = Xp[:, :F]
+        del Xp
+    ld = args.ld or F
+    outs = [torch.empty((g.n, ld), dtype=torch.float32, device="cuda")[:, :F] for _ in range(K)]
     small = g.n * F * 4 <= 126e6
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
     stream = torch.cuda.current_stream()
@@ -443,7 +452,7 @@ def main():
     seg_launch_ms = seg_ms / max(1, seg_launches)
     achieved = gather_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9
     traffic = (profiled_traffic(w.name) if args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1
-               and not args.no_bulk_copy and not args.feat_dim and args.op < 0 else None)
+               and not args.no_bulk_copy and not args.feat_dim and args.op < 0 and not args.ld else None)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": traffic,
                 "dram_achieved": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9,
@@ -525,7 +534,7 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
                 "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": dict(workload_config(w, g, info), parallelism="column shards" if sharded else "replicas", cuda_graph=bool(args.cuda_graph)), "clocks": clocks.summary(), "e2e": e2e,
+                "config": dict(workload_config(w, g, info), parallelism="column shards" if sharded else "replicas", cuda_graph=bool(args.cuda_graph), leading_dim=ld), "clocks": clocks.summary(), "e2e": e2e,
                 "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
                 "plan_build_ms": plan_ms, "input_generation_s": gen_s,
                 # the same metric if every step also rebuilt the plan (degrees, scales, Eq. 12, edge blocks, segments)

@@ -167,8 +167,10 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
         inflight[st] = false;
     }
     bool failed = false;
-    const bool on = lane < a.f4;  // lanes beyond the row's width re-read column 0 and never store
-    const uint32_t lane_off = on ? 16u * lane : 0u;
+    // Lanes beyond the row's width never store; they re-read the row's last float4, the address their
+    // quarter-warp already reads (one broadcast), so they add no shared-memory wavefront.
+    const bool on = lane < a.f4;
+    const uint32_t lane_off = on ? 16u * lane : rb - 16u;
     const unsigned lt_mask = (1u << lane) - 1u;
 
     const int64_t W = (int64_t)gridDim.x * nwarps;
@@ -249,6 +251,38 @@ __global__ void __launch_bounds__(kTmaMaxWarps * 32, 1)
             phase[st] ^= 1u;
             inflight[st] = false;
             const unsigned char* base = my_smem + st * stage_bytes + lane_off;
+            if (kTmaRows == 2 * kTmaStep && m.cnt == kTmaRows && m.ends == 0) {
+                // A full chunk inside one row (most of a hub's chunks): its two steps are summed side by
+                // side, four rows of each at a time, so that four independent chains of adds are in
+                // flight instead of two.  Each step's sum is still the plain chain over its 8 rows and
+                // the two sums still join the compensated sum in edge order: same bits as the loop below.
+                Quad acc2 = quad_zero();
+#pragma unroll
+                for (int h = 0; h < kTmaStep; h += 4) {
+                    Quad xa[4], xb[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        xa[u] = quad_load(base + ((h + u) >> 2) * group_bytes + ((h + u) & 3) * rb);
+                        xb[u] = quad_load(base + ((kTmaStep + h + u) >> 2) * group_bytes + ((kTmaStep + h + u) & 3) * rb);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (OP == GNNPRE_OP_SAGE_MEAN) {
+                            quad_add(acc, xa[u]);
+                            quad_add(acc2, xb[u]);
+                        } else {
+                            quad_fma(acc, __shfl_sync(kFull, m.w, h + u), xa[u]);
+                            quad_fma(acc2, __shfl_sync(kFull, m.w, kTmaStep + h + u), xb[u]);
+                        }
+                    }
+                }
+                quad_kahan(tot, cmp, acc);
+                quad_kahan(tot, cmp, acc2);
+                acc = quad_zero();
+                open = true;
+                __syncwarp();
+                return;
+            }
             for (int t0 = 0; t0 < m.cnt; t0 += kTmaStep) {
                 Quad x[kTmaStep];
 #pragma unroll

@@ -28,20 +28,25 @@ def B():
 @pytest.mark.parametrize("op", (0, 1, 2))
 def test_static_hop_matches_planned_hop_twice_in_a_row(B, op):
     """Two calls back to back with different inputs: the second must not see anything the first left
-    in the shared scratch array.  Compared with the fp64 oracle at the tolerance of the parity tests;
-    the graph has isolated nodes and hubs far longer than a segment."""
+    in the shared scratch array.  Each result is compared with the hop that the planned entry point
+    (gnnpre_build_plan + gnnpre_propagate) gives for the same inputs, and with the fp64 oracle, both at
+    the tolerance of the parity tests; the graph has isolated nodes and hubs far longer than a segment."""
     g = gi.rmat(20000, 300000, 21, directed_candidates=True)
     drp, dci = g.rowptr.cuda(), g.colidx.cuda()
     rp, ci = g.rowptr.numpy(), g.colidx.numpy()
     for F in (100, 16):
+        plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=0.1)
         for seed in (1, 2):
             X = gi.normal_matrix(g.n, F, seed, device="cuda")
             want = orc.propagate(op, 0.1, rp, ci, to_np(X), 1)[0]
+            planned, _ = B.gnnpre_propagate(plan, X, 1)
             buf = torch.full((g.n, F + 4), -5.0, device="cuda")
             got = B.gnnpre_hop_static(drp, dci, op, X, buf[:, :F], gin_eps=0.1)
             torch.cuda.synchronize()
+            assert hop_error(to_np(got), to_np(planned[0]).astype(np.float64)) <= TOL
             assert hop_error(to_np(got), want) <= TOL
             assert bool((buf[:, F:] == -5.0).all())
+        plan.close()
 
 
 def test_static_hop_edge_cases_and_limits(B):
