@@ -379,6 +379,8 @@ def main():
     plan_ms = (time.perf_counter() - t0) * 1e3
     info = plan.info()
     m = info["nnz_tilde"]
+    if not args.ld and F % 4:
+        args.ld = (F + 3) // 4 * 4  # the library wants leading dimensions that are multiples of 4 floats
     if args.ld:  # rows padded to the given leading dimension: strided views, the library takes ldx / ldo
         assert args.ld >= F and args.ld % 4 == 0 and not (args.shard == "columns" and world > 1)
         Xp = torch.zeros((g.n, args.ld), dtype=torch.float32, device="cuda")
@@ -469,9 +471,9 @@ def main():
     e2e = None
     if not args.no_e2e and rank == 0:
         try:
-            Xh = torch.empty((g.n, F), dtype=torch.float32, pin_memory=True)
+            Xh = torch.zeros((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F]
             Xh.copy_(X)
-            outs_h = [torch.empty((g.n, F), dtype=torch.float32, pin_memory=True) for _ in range(K)]
+            outs_h = [torch.empty((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F] for _ in range(K)]
             if w.streamed:  # the graph lives in pinned host memory too; its edge blocks are streamed
                 rp_e2e, ci_e2e = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
             else:
@@ -498,7 +500,7 @@ def main():
             e2e["blocks"] = hinfo["b"]
             e2e["structure_on_host"] = bool(hinfo["structure_mem"])
             # same bits are expected only when both plans cut the edge list the same way
-            comparable = hinfo["c"] == 1 and hinfo["segment_edges"] == info["segment_edges"]
+            comparable = hinfo["c"] == 1 and hinfo["b"] == info["b"] and hinfo["segment_edges"] == info["segment_edges"]
             same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if comparable else None
             e2e["bitwise_equal_to_resident"] = same
             e2e["max_abs_diff_to_resident"] = max(float((o.cpu() - h).abs().max()) for o, h in zip(outs, outs_h))
@@ -528,7 +530,7 @@ def main():
     # ---------------- the oracle on this machine's host cores, bounded sample (rank 0, one GPU only)
     cpu = None
     if not args.no_cpu_baseline and rank == 0 and world == 1:
-        cpu, _ = oracle_sample(w, g.to("cpu"), X.cpu().numpy(), args.cpu_seconds)
+        cpu, _ = oracle_sample(w, g.to("cpu"), np.ascontiguousarray(X.cpu().numpy()), args.cpu_seconds)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

@@ -10,6 +10,12 @@ synthetic stand-ins, because the public datasets are not available offline.
   c4  R-MAT, 2,449,029 nodes, 61,859,140 undirected edges, F=100, K=3, SAGE, b=32
   c5  R-MAT, 111,059,956 nodes, 807,842,936 undirected edges, F=128, K=2, GCN, streamed
 
+and two more with the node count, edge count and feature width of the two wide-feature datasets of
+that table (rows of 2,000 and 2,408 bytes):
+
+  flickr  R-MAT,  89,250 nodes,    899,756 undirected edges, F=500, K=2, GCN
+  reddit  R-MAT, 232,965 nodes, 11,606,919 undirected edges, F=602, K=2, GCN
+
 This module holds no arithmetic of the propagation method itself.
 """
 from __future__ import annotations
@@ -49,6 +55,8 @@ WORKLOADS = {
     "c4": Workload("c4", "rmat", 2449029, 61859140, False, 100, 3, OP_SAGE, 32, BASE_SEED + 3),
     "c5": Workload("c5", "rmat", 111059956, 807842936, False, 128, 2, OP_GCN, 0, BASE_SEED + 4,
                    streamed=True),
+    "flickr": Workload("flickr", "rmat", 89250, 899756, False, 500, 2, OP_GCN, 0, BASE_SEED + 5),
+    "reddit": Workload("reddit", "rmat", 232965, 11606919, False, 602, 2, OP_GCN, 0, BASE_SEED + 6),
 }
 
 

@@ -347,11 +347,16 @@ int32_t auto_segment_edges(int64_t slab_width, int64_t m, bool bulk_copy, int nu
         return p;
     }
     // about 32 Ki gathered floats per segment, but short enough that every SM's 2048 threads get a
-    // segment per lane group; a power of two between 32 and 4096 edges
+    // segment per lane group; a power of two between 32 and 4096 edges.  Rows wider than 256 floats
+    // get at least 128 edges per segment (256 when the graph still leaves a thousand edges per lane
+    // group): with shorter ones most rows are cut and adding up their parts costs more than the
+    // segments save (F = 602, 23 M edges: 17.0 ms per two hops at 32 edges, 13.5 ms at 256).
     const int64_t f4 = std::min<int64_t>(std::max<int64_t>(slab_width, 4), 512) / 4;
     const int64_t lanes = f4 <= 4 ? 4 : f4 <= 8 ? 8 : f4 <= 16 ? 16 : 32;
     const int64_t groups = (int64_t)std::max(num_sms, 1) * (2048 / lanes);
-    const int64_t L = std::min<int64_t>(32768 / std::max<int64_t>(slab_width, 4), m / groups);
+    int64_t by_width = 32768 / std::max<int64_t>(slab_width, 4);
+    if (by_width < 128) by_width = m / groups >= 1024 ? 256 : 128;
+    const int64_t L = std::min<int64_t>(by_width, m / groups);
     int32_t p = 32;
     while ((int64_t)p * 2 <= L && p < 4096) p *= 2;
     return p;

@@ -436,7 +436,7 @@ int launch_segments_tma_width(const gnnpre_plan* P, const SegArgs& a, cudaStream
     return GNNPRE_OK;
 }
 
-// The two widths of the paper's datasets (F = 100, F = 128) get kernels with the row size compiled in.
+// Rows (or column tiles) of 100 and of 128 columns get kernels with the row size compiled in.
 template <int OP, bool HAS_EMPTY>
 int launch_segments_tma_op(const gnnpre_plan* P, const SegArgs& a, cudaStream_t st) {
     const int ep = epilogue_of(a.tp);
@@ -487,16 +487,33 @@ Teleport teleport_of(const gnnpre_plan* P, const HopArgs& h, int32_t f0) {
 
 }  // namespace
 
-// Rows of 68..128 columns (17..32 float4) go through the bulk-copy kernel unless the plan says otherwise.
-bool uses_bulk_copy(const gnnpre_plan* P, int32_t width) {
+namespace {
+
+// A column tile of 68..128 columns (17..32 float4) goes through the bulk-copy kernel unless the plan says otherwise.
+bool tile_uses_bulk_copy(const gnnpre_plan* P, int32_t width) {
     const int32_t f4 = width / 4;
     return !(P->flags & GNNPRE_FLAG_NO_BULK_COPY) && f4 > 16 && f4 <= 32 && tma_warps(f4) >= 2;
 }
 
+// Columns one segment launch covers.  Rows wider than 256 columns are cut into 128-column tiles for the bulk-copy
+// kernel: the register kernel holds only two such rows per lane in flight (F = 602 on 23 M edges: 8.4 TB/s of
+// gathered bytes for its 512-column tile against 11 TB/s for the copy engine on the rest of the row).
+int32_t segment_tile_width(const gnnpre_plan* P, int32_t width) {
+    return width > 256 && tile_uses_bulk_copy(P, 128) ? 128 : kMaxTile;
+}
+
+}  // namespace
+
+// Whether a slab of this width is (mostly) summed by the bulk-copy kernel; the plan sizes its segments for it.
+bool uses_bulk_copy(const gnnpre_plan* P, int32_t width) {
+    return tile_uses_bulk_copy(P, std::min(width, segment_tile_width(P, width)));
+}
+
 int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int64_t seg_hi, cudaStream_t st) {
     if (seg_hi <= seg_lo) return GNNPRE_OK;
-    for (int32_t f0 = 0; f0 < h.width; f0 += kMaxTile) {
-        const int32_t w = std::min<int32_t>(kMaxTile, h.width - f0);
+    const int32_t tile = segment_tile_width(P, h.width);
+    for (int32_t f0 = 0; f0 < h.width; f0 += tile) {
+        const int32_t w = std::min<int32_t>(tile, h.width - f0);
         SegArgs a;
         a.segs = P->segments.p;
         a.seg_lo = seg_lo;
@@ -515,7 +532,7 @@ int launch_segments(const gnnpre_plan* P, const HopArgs& h, int64_t seg_lo, int6
         a.f4 = w / 4;
         a.diag_weight = 1.0f + P->gin_eps;
         a.tp = teleport_of(P, h, f0);
-        if (uses_bulk_copy(P, w)) GNNPRE_TRY(launch_segments_tma(P, a, st));
+        if (tile_uses_bulk_copy(P, w)) GNNPRE_TRY(launch_segments_tma(P, a, st));
         else if (a.f4 <= 4) GNNPRE_TRY((launch_segments_shape<4, 1, 4>(P, a, st)));
         else if (a.f4 <= 8) GNNPRE_TRY((launch_segments_shape<8, 1, 8>(P, a, st)));
         else if (a.f4 <= 16) GNNPRE_TRY((launch_segments_shape<16, 1, 8>(P, a, st)));
@@ -604,6 +621,8 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
                 h.zsum_first = k == 0;
             }
             const int tiles = (h.width + kMaxTile - 1) / kMaxTile;
+            const int seg_tile = segment_tile_width(P, h.width);
+            const int seg_tiles = (h.width + seg_tile - 1) / seg_tile;
             rc = launch_zero_empty_rows(P, h, st);
             launches += P->num_empty ? 1 : 0;
             const bool per_block = (P->flags & GNNPRE_FLAG_LAUNCH_PER_BLOCK) != 0;
@@ -617,8 +636,8 @@ int propagate_resident(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, f
                     rc = mark(seg_ev);
                     if (rc == GNNPRE_OK) rc = launch_segments(P, h, seg_lo, seg_hi, st);
                     if (rc == GNNPRE_OK) rc = mark(seg_ev);
-                    launches += tiles;
-                    seg_launches += tiles;
+                    launches += seg_tiles;
+                    seg_launches += seg_tiles;
                 }
                 if (rc == GNNPRE_OK && fix_hi > fix_lo) {
                     rc = launch_fixups(P, h, fix_lo, fix_hi, st);

@@ -125,3 +125,40 @@ def test_first_dense_stage_at_config4_size_sampled(B):
     assert float(Y[1].min()) >= 0.0 and float(Y[2].min()) >= 0.0 and float(Y[0].min()) < 0.0
     Z = B.gnnpre_lc_first_layer(hops[:1], None, Wt)
     assert torch.equal(Z[0][order.long()[:100000]], Y[0][:100000])
+
+
+@pytest.mark.parametrize("name", ("flickr", "reddit"))
+def test_wide_feature_dataset_shapes_full_size(B, name):
+    """The two wide-feature rows of the paper's dataset table as seeded R-MAT stand-ins (89,250 nodes / 899,756
+    edges / F=500 and 232,965 nodes / 11,606,919 edges / F=602), GCN, K=2, whole graph resident.  F=602 is not a
+    multiple of 4: the matrices carry a leading dimension of 604.  Degrees bit-exact; every hop against the fp64
+    chain; hop 1 floor-free on sampled rows (random and the highest degrees); the sum GCN conserves on a symmetric
+    graph, sum_i sqrt(d_i + 1) X_k[i, f], unchanged from hop to hop."""
+    w = gi.WORKLOADS[name]
+    g = gi.make_graph(w, device="cuda")
+    F, K = w.feat_dim, w.hops
+    ld = (F + 3) // 4 * 4
+    X = gi.make_features(w, device="cuda", ld=ld)
+    assert (g.n, g.nnz) == (w.n, 2 * w.m)
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F)
+    outs = [torch.full((g.n, ld), float("nan"), device="cuda")[:, :F] for _ in range(K)]
+    B.gnnpre_propagate(plan, X, K, outs)
+    torch.cuda.synchronize()
+    rp, ci = to_np(g.rowptr), to_np(g.colidx)
+    deg, _, _ = B.gnnpre_plan_scales(plan)
+    np.testing.assert_array_equal(deg.numpy(), orc.degrees(rp))
+    X_np = np.ascontiguousarray(to_np(X))
+    want = orc.propagate(w.op, 0.0, rp, ci, X_np, K)
+    rng = np.random.default_rng(7)
+    rows = np.unique(np.concatenate([rng.integers(0, g.n, 2048), np.argsort(deg.numpy())[-64:]]))
+    sq = torch.sqrt(torch.from_numpy(deg.numpy()).cuda().double() + 1.0)
+    prev = X
+    for k in range(K):
+        got = np.ascontiguousarray(to_np(outs[k]))
+        assert hop_error(got, want[k]) <= TOL
+        if k == 0:
+            assert backward_error(w.op, 0.0, rp, ci, X_np, got, rows) <= TOL
+        a, b_ = sq @ outs[k].double(), sq @ prev.double()
+        assert float(((a - b_).abs() / (sq @ prev.double().abs())).max()) <= 1e-6
+        prev = outs[k]
+    plan.close()

@@ -321,10 +321,14 @@ def test_streamed_pageable_host_memory_and_check_against_oracle(B):
 
 
 @pytest.mark.parametrize("op", OPS)
-@pytest.mark.parametrize("F", [68, 100, 128])
+@pytest.mark.parametrize("F", [68, 100, 128, 300, 516])
 def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
-    """Rows of 68..128 columns are staged through shared memory by the copy engine; the summation
-    order is the register kernel's, so the two agree bit for bit (and both agree with the oracle)."""
+    """Rows of 68..128 columns are staged through shared memory by the copy engine; the summation order is that
+    of the register kernel for such rows (plain sums over steps of 8 edges), so the two agree bit for bit (and both
+    agree with the oracle).  Rows wider than 256 columns are cut into 128-column tiles for the copy engine
+    (300 = 128 + 128 + a 44-column tile left to the register kernel; 516 = four tiles + 4 columns); the register
+    kernel for rows that wide sums over steps of 2 edges, so there the two paths agree to rounding only and each
+    is checked against the oracle."""
     g = gi.rmat(30000, 400000, 17, directed_candidates=True)
     drp, dci = dev(g)
     X = gi.normal_matrix(g.n, F, 9, device="cuda")
@@ -336,7 +340,11 @@ def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
             res.append(outs)
             plan.close()
         for k in range(2):
-            assert torch.equal(res[0][k], res[1][k]), (b, seg, k)
+            if F <= 128:
+                assert torch.equal(res[0][k], res[1][k]), (b, seg, k)
+        if F > 128:
+            check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[1])
+            check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[0])
     check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[0])
 
 
