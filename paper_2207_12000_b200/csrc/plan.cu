@@ -585,8 +585,10 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
         // Host-resident operands: Eq. 12's model charges every block product the same, but with copies
         // overlapped a second slab lets the upload of X and the first hop's kernels run side by side.
         // Two slabs are used when the budget alone asks for one and the row pieces stay >= 256 bytes
-        // (narrower strided pieces travel the host link below full speed).
-        if (opts->force_col_slabs == 0 && opts->operands_mem == GNNPRE_MEM_HOST && c == 1 && F >= 128 && F % 8 == 0)
+        // (narrower strided pieces travel the host link below full speed); below 256 columns only for
+        // two equal slabs, so that the pieces also start on 128-byte lines.
+        if (opts->force_col_slabs == 0 && opts->operands_mem == GNNPRE_MEM_HOST && c == 1 && F >= 128 &&
+            (F % 8 == 0 || F >= 256))
             c = 2;
         // Likewise a single edge block would hold every output row back until the whole hop is done;
         // eight blocks let finished rows leave for the host while the rest of the hop computes.

@@ -162,3 +162,13 @@ def test_wide_feature_dataset_shapes_full_size(B, name):
         assert float(((a - b_).abs() / (sq @ prev.double().abs())).max()) <= 1e-6
         prev = outs[k]
     plan.close()
+    if name == "flickr":  # the same call through pinned host buffers: two column slabs of 252 and 248 columns
+        hplan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, operands_mem=B.GNNPRE_MEM_HOST)
+        assert hplan.info()["c"] == 2
+        Xh = torch.zeros((g.n, ld), dtype=torch.float32).pin_memory()[:, :F]
+        Xh.copy_(X)
+        outs_h = [torch.full((g.n, ld), float("nan")).pin_memory()[:, :F] for _ in range(K)]
+        B.gnnpre_propagate(hplan, Xh, K, outs_h)
+        for k in range(K):
+            assert hop_error(np.ascontiguousarray(outs_h[k].numpy()), want[k]) <= TOL
+        hplan.close()
