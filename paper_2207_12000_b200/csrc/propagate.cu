@@ -498,8 +498,27 @@ bool tile_uses_bulk_copy(const gnnpre_plan* P, int32_t width) {
 // Columns one segment launch covers.  Rows wider than 256 columns are cut into 128-column tiles for the bulk-copy
 // kernel: the register kernel holds only two such rows per lane in flight (F = 602 on 23 M edges: 8.4 TB/s of
 // gathered bytes for its 512-column tile against 11 TB/s for the copy engine on the rest of the row).
+// Rows of 132..256 columns go the same way, as two equal tiles, once a 128-column tile of X no longer fits the
+// L2 (2.4 M nodes, 124 M edges, F = 256: 11.9 ms per hop-launch on the register kernel plus 1.6 ms of fix-ups for
+// its 128-edge segments, against 2 x 4.7 ms); while it fits, the register kernel's four rows per lane are the
+// faster path (169 K nodes, F = 256: 0.25 ms against 2 x 0.15 ms).
+int64_t l2_cache_bytes() {
+    static int64_t cached = -1;
+    if (cached < 0) {
+        int dev = 0, bytes = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&bytes, cudaDevAttrL2CacheSize, dev) != cudaSuccess || bytes <= 0)
+            bytes = 126 << 20;
+        cached = bytes;
+    }
+    return cached;
+}
+
 int32_t segment_tile_width(const gnnpre_plan* P, int32_t width) {
-    return width > 256 && tile_uses_bulk_copy(P, 128) ? 128 : kMaxTile;
+    if (!tile_uses_bulk_copy(P, 128)) return kMaxTile;
+    if (width > 256) return 128;
+    if (width > 128 && P->n * 512 > l2_cache_bytes()) return 4 * ((width / 4 + 1) / 2);
+    return kMaxTile;
 }
 
 }  // namespace

@@ -348,6 +348,28 @@ def test_bulk_copy_kernel_matches_register_kernel_bitwise(B, op, F):
     check_all_hops(op, EPS, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), res[0])
 
 
+def test_two_tile_rows_on_a_graph_larger_than_the_cache(B):
+    """Rows of 132..256 columns are cut into two equal tiles for the copy engine once a 128-column tile of X no
+    longer fits the L2 (here 400,000 nodes: 205 MB per tile; F = 200 gives two tiles of 100 columns, F = 252 two of
+    128 and 124).  Checked against the oracle, and against the register kernel to rounding."""
+    g = gi.rmat(400000, 3000000, 23, directed_candidates=True)
+    drp, dci = dev(g)
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    for op, F in ((1, 200), (0, 252)):
+        X = gi.normal_matrix(g.n, F, 12, device="cuda")
+        res = []
+        for flags in (0, B.GNNPRE_FLAG_NO_BULK_COPY):
+            plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, flags=flags)
+            outs, st = B.gnnpre_propagate(plan, X, 2, want_stats=True)
+            torch.cuda.synchronize()
+            res.append((outs, st.kernel_launches, plan.info()["segment_edges"]))
+            plan.close()
+        assert res[0][2] >= 256 and res[0][1] > res[1][1]  # long segments, two segment launches per hop
+        check_all_hops(op, EPS, rp, ci, to_np(X), res[0][0])
+        for k in range(2):
+            assert hop_error(to_np(res[0][0][k]), to_np(res[1][0][k]).astype(np.float64)) <= TOL
+
+
 # ------------------------------------------------------------------ the normalised adjacency itself
 
 @pytest.mark.parametrize("op", OPS)
