@@ -65,6 +65,10 @@ def parse():
                     help="--stage lc: tf32 operands, or every operand split into two tf32 numbers (fp32-like accuracy)")
     ap.add_argument("--e2e-col-slabs", type=int, default=0, help="column slabs c of the host-buffer run (0 = the library's choice)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="default run only: skip the compact records of configurations 1, 2, 3 (a corner) and 5")
+    ap.add_argument("--c5-scale", type=int, default=2,
+                    help="divisor of configuration 5's nodes and edges in the default run's streamed record")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     return ap.parse_args()
 
@@ -132,10 +136,16 @@ def profiled_traffic(workload_name):
     h = re.search(r"kernel_source_sha256:\s*([0-9a-f]{64})", text)
     if not t or not h:
         return None
+    return int(t.group(1)) if kernel_source_hash() == h.group(1) else None
+
+
+def kernel_source_hash():
+    """sha256 over the files that hold the segment kernels (what an ncu capture of them depends on)."""
+    import hashlib
     cur = hashlib.sha256()
-    for f in ("propagate.cu", "segments_tma.cuh"):
+    for f in ("segments.cuh", "segments_tma.cuh"):
         cur.update(open(os.path.join(ROOT, "paper_2207_12000_b200", "csrc", f), "rb").read())
-    return int(t.group(1)) if cur.hexdigest() == h.group(1) else None
+    return cur.hexdigest()
 
 
 def profiled_traffic_lc(rows_per_launch):
@@ -181,15 +191,17 @@ def byte_model(n, m, F):
     return gather, least
 
 
-def oracle_sample(w, g_cpu, X_cpu, target_seconds):
-    """Times the CPU oracle, as it stands, on a row range of hop 1 sized for about target_seconds."""
+def oracle_sample(w, g_cpu, X_cpu, target_seconds, got=None):
+    """Times the CPU oracle, as it stands, on a row range of hop 1 sized for about target_seconds.  `got` maps a
+    label to hop 1 as the CUDA path computed it (anything indexable by a row range that gives a numpy array):
+    the rows the oracle has just computed are then compared with it, floor-free, |g - o| / (|A^| |x|)."""
     import oracle as orc
     rp, ci = g_cpu.rowptr.numpy(), g_cpu.colidx.numpy()
     n = g_cpu.n
     diag = 0 if w.op == gi.OP_SAGE else 1
     probe_rows = max(1, n // 256)
     t0 = time.perf_counter()
-    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(probe_rows), want_abs=False)
+    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(probe_rows))
     t_probe = time.perf_counter() - t0
     probe_edges = int(rp[probe_rows]) + diag * probe_rows
     rate = probe_edges / max(t_probe, 1e-6)
@@ -198,11 +210,21 @@ def oracle_sample(w, g_cpu, X_cpu, target_seconds):
     rows = n if want_edges >= total_edges else int(np.searchsorted(rp, want_edges))
     rows = max(1, min(n, rows))
     t0 = time.perf_counter()
-    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(rows), want_abs=False)
+    y, scale = orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(rows))
     t = time.perf_counter() - t0
     edges = int(rp[rows]) + diag * rows
-    return {"value": edges * X_cpu.shape[1] / t, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
-            "sample": f"hop 1 of {w.name} on rows [0, {rows}) = {edges} of {total_edges} edges, {t:.2f} s"}, t
+    out = {"value": edges * X_cpu.shape[1] / t, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
+           "sample": f"hop 1 of {w.name} on rows [0, {rows}) = {edges} of {total_edges} edges, {t:.2f} s"}
+    if got:
+        nz = scale > 0
+        parity = {"rows": rows, "tolerance": 1e-5, "measure": "max |gpu - oracle| / (|A^| |X|) over the sampled rows of hop 1"}
+        for label, hop1 in got.items():
+            g = np.asarray(hop1[0:rows], dtype=np.float64)
+            err = float((np.abs(g - y)[nz] / scale[nz]).max(initial=0.0))
+            exact_zero = bool((g[~nz] == 0).all())
+            parity[label] = {"max_backward_error": err, "ok": bool(err <= 1e-5 and exact_zero)}
+        out["parity"] = parity
+    return out, t
 
 
 def run_reference(args, w):
@@ -323,6 +345,217 @@ def run_lc_stage(args, w):
     print(json.dumps(line))
 
 
+_LINK = {}
+
+
+def host_link_peak():
+    """The host link's ceiling measured in this process: one 1 GiB pinned copy per direction, best of 3."""
+    if _LINK:
+        return dict(_LINK)
+    pin = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
+    devb = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    for name, dst, src in (("h2d_gbs", devb, pin), ("d2h_gbs", pin, devb)):
+        best = 0.0
+        for _ in range(3):
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            dst.copy_(src, non_blocking=True)
+            torch.cuda.synchronize()
+            best = max(best, (1 << 30) / (time.perf_counter() - t0) / 1e9)
+        _LINK[name] = best
+    del pin, devb
+    return dict(_LINK)
+
+
+def link_record(stats, seconds):
+    """Achieved host-link rate of a streamed call against the measured ceiling of its busier direction."""
+    link = host_link_peak()
+    moved = max(stats.h2d_bytes, stats.d2h_bytes)
+    link["achieved_gbs"] = moved / seconds / 1e9
+    link["direction"] = "d2h" if stats.d2h_bytes >= stats.h2d_bytes else "h2d"
+    link["frac"] = link["achieved_gbs"] / link[link["direction"] + "_gbs"]
+    return link
+
+
+def time_resident(B, plan, X, K, outs, steps, warmup, flush, stream, graph=None, barrier=None, sampler_index=None):
+    """Device-resident timing of `steps` gnnpre_propagate calls with CUDA events on the launching stream.
+    Pass 1 times the calls as a user makes them (asynchronous): ms per step.  Pass 2 repeats them with the
+    library's per-launch events on: duration of the segment kernel.  Returns a dict."""
+    barrier = barrier or torch.cuda.synchronize
+
+    def step(want_stats, start=None):
+        if flush is not None:
+            flush.fill_(1)  # L2 flush between iterations, outside the timed interval
+        if start is not None:
+            start.record(stream)
+        if graph is not None and not want_stats:
+            graph.replay()
+            return None
+        _, st = B.gnnpre_propagate(plan, X, K, outs, stream=stream, want_stats=want_stats)
+        return st
+
+    for _ in range(max(3, warmup)):
+        step(False)
+    barrier()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    seg_ms, seg_launches, launches, st = 0.0, 0, 0, None
+    sampler = ClockSampler(sampler_index) if sampler_index is not None else None
+    if sampler:
+        sampler.__enter__()
+    barrier()
+    for a, b_ in ev:
+        step(False, start=a)
+        b_.record(stream)
+    barrier()
+    for a, b_ in ev2:
+        st = step(True, start=a)
+        b_.record(stream)
+        seg_ms += st.segments_ms
+        seg_launches += st.segments_launches
+        launches += st.kernel_launches
+    barrier()
+    if sampler:
+        sampler.__exit__()
+    step_ms = [a.elapsed_time(b_) for a, b_ in ev]
+    return {"total_ms": float(sum(step_ms)), "ms_per_step": float(sum(step_ms)) / steps,
+            "seg_ms": seg_ms, "seg_launches": seg_launches, "launches": launches,
+            "pass2_ms": float(sum(a.elapsed_time(b_) for a, b_ in ev2)),
+            "hop_ms": [float(st.hop_ms[k]) for k in range(K)], "clocks": sampler.summary() if sampler else None}
+
+
+def time_ceiling(B, plan, X, flush, stream, reps=10):
+    """Average duration of the fetch-only yardstick (gnnpre_gather_ceiling: one hop's gathers, rows summed
+    plainly, nothing stored), timed like a hop: CUDA events, L2 flushed before each when the hop runs flushed."""
+    sink = B.gnnpre_gather_ceiling(plan, X, stream=stream)
+    for _ in range(2):
+        B.gnnpre_gather_ceiling(plan, X, sink, stream=stream)
+    ms = []
+    for _ in range(reps):
+        if flush is not None:
+            flush.fill_(1)
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        B.gnnpre_gather_ceiling(plan, X, sink, stream=stream)
+        b_.record(stream)
+        torch.cuda.synchronize()
+        ms.append(a.elapsed_time(b_))
+    if B.gnnpre_plan_status(plan, stream) != 0:
+        raise RuntimeError("a bounded wait ran out inside the gather-ceiling kernel")
+    return float(np.mean(ms))
+
+
+def compact_resident_record(B, w, steps=20, blocks=None):
+    """One device-resident workload measured like the headline one, reported as a compact record: ms per step
+    (all K hops), the segment kernel per hop, and the fetch-only yardstick beside it."""
+    g = gi.make_graph(w, device="cuda")
+    X = gi.make_features(w, device="cuda")
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    K, F = w.hops, w.feat_dim
+    b = w.blocks if blocks is None else blocks
+    plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, gin_eps=w.gin_eps, force_blocks=b,
+                               force_col_slabs=1 if b else 0)
+    info = plan.info()
+    m = info["nnz_tilde"]
+    outs = [torch.empty((g.n, F), dtype=torch.float32, device="cuda") for _ in range(K)]
+    small = g.n * F * 4 <= 126e6
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda") if small else None
+    stream = torch.cuda.current_stream()
+    t = time_resident(B, plan, X, K, outs, steps, 3, flush, stream)
+    ceil_ms = time_ceiling(B, plan, X, flush, stream)
+    seg_ms_per_hop = t["seg_ms"] / (steps * K)
+    gather_b, least_b = byte_model(g.n, m, F)
+    rec = {"workload": workload_config(w, g, info)["workload"], "blocks": info["b"], "segment_edges": info["segment_edges"],
+           "l2": "flushed between steps" if small else "inputs larger than L2",
+           "ms_per_step": t["ms_per_step"], "value": K * m * F / (t["ms_per_step"] * 1e-3), "unit": UNIT,
+           "segment_kernel_ms_per_hop": seg_ms_per_hop,
+           "segment_launches_per_hop": t["seg_launches"] / (steps * K),
+           "gather_ceiling_ms_per_hop": ceil_ms,
+           "frac_of_gather_ceiling": ceil_ms / seg_ms_per_hop if seg_ms_per_hop > 0 else None,
+           "gather_model_gbs": gather_b / (seg_ms_per_hop * 1e-3) / 1e9,
+           "gpu_launches_per_step": t["launches"] / steps}
+    plan.close()
+    return rec
+
+
+def streamed_run(B, w, g, X_dev, args, reps, blocks, col_slabs, ld=None):
+    """The same metric through the C ABI with HOST buffers: X and every hop in pinned host memory (the graph too
+    for streamed workloads), copies inside the timed region.  Returns (record, hop-1 host tensor or None)."""
+    K, F = w.hops, w.feat_dim
+    ld = ld or F
+    if X_dev.is_cuda:
+        Xh = torch.zeros((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F]
+        Xh.copy_(X_dev)
+    else:
+        Xh = X_dev  # already in pinned host memory
+    outs_h = [torch.empty((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F] for _ in range(K)]
+    if w.streamed:  # the graph lives in pinned host memory too
+        rp, ci = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
+    else:
+        rp, ci = g.rowptr, g.colidx
+    plan = B.gnnpre_build_plan(rp, ci, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks, force_col_slabs=col_slabs,
+                               segment_edges=args.segment_edges, budget_bytes=int(args.budget_gb * 1e9),
+                               operands_mem=B.GNNPRE_MEM_HOST)
+    for _ in range(2):
+        B.gnnpre_propagate(plan, Xh, K, outs_h)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        _, st = B.gnnpre_propagate(plan, Xh, K, outs_h, want_stats=True)
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / reps
+    info = plan.info()
+    rec = {"value": K * info["nnz_tilde"] * F / dt, "unit": UNIT, "h2d_bytes_per_step": int(st.h2d_bytes),
+           "d2h_bytes_per_step": int(st.d2h_bytes), "ms_per_step": dt * 1e3, "steps": reps,
+           "col_slabs": info["c"], "blocks": info["b"], "structure_on_host": bool(info["structure_mem"]),
+           "schedule": ("resident", "equal column slabs", "narrow-first column panels")[st.schedule],
+           "upload_slabs": int(st.upload_slabs), "startup_ms": float(st.startup_ms), "drain_ms": float(st.drain_ms),
+           "host_link": link_record(st, dt), "segment_edges": info["segment_edges"]}
+    plan.close()
+    return rec, outs_h, Xh
+
+
+def c5_streamed_record(B, args):
+    """Configuration 5, scaled to what the host's memory holds, as the paper's streamed setting: graph, X and
+    both hop outputs in pinned host memory, default budget.  Reports the host-link fraction and checks the
+    outputs it timed against the oracle on a bounded row sample (part of the CPU-baseline leg)."""
+    w = gi.scaled(gi.WORKLOADS["c5"], args.c5_scale)
+    g = gi.make_graph(w, device="cuda")
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    Xh = gi.normal_matrix(w.n, w.feat_dim, w.seed, device="cuda", pin=True)
+    torch.cuda.synchronize()
+    torch.cuda.empty_cache()
+    rec, outs_h, Xh = streamed_run(B, w, g, Xh, args, reps=3, blocks=0, col_slabs=0)
+    rec["workload"] = (f"{w.name}: rmat graph, {g.n} nodes, {g.nnz} directed nnz, F={w.feat_dim}, K={w.hops}, op=gcn_sym; "
+                       "graph, X and hop outputs in pinned host memory")
+    rec["scale_note"] = (f"configuration 5 at 1/{args.c5_scale} of its nodes and edges: at full size X and two hop outputs alone "
+                         "are 171 GB of pinned memory, more than the host of this machine has beside the generator")
+    if not args.no_cpu_baseline:
+        cpu, _ = oracle_sample(w, g.to("cpu"), Xh.numpy(), min(args.cpu_seconds, 4.0), got={"streamed": outs_h[0].numpy()})
+        rec["cpu_baseline"] = cpu
+        rec["parity_checked"] = bool(cpu["parity"]["streamed"]["ok"])
+    del outs_h, Xh
+    return rec
+
+
+def configs_object(B, args):
+    """Compact records of the other configurations (1, 2, a corner of 3's sweep, and 5 streamed), so that one
+    default run carries a measured line for each of the five."""
+    import dataclasses
+    out = {}
+    out["c1"] = compact_resident_record(B, gi.WORKLOADS["c1"], steps=50)
+    out["c2"] = compact_resident_record(B, gi.WORKLOADS["c2"], steps=20)
+    c3 = gi.WORKLOADS["c3"]
+    for op, opname in ((gi.OP_GCN, "gcn"), (gi.OP_SAGE, "sage")):
+        for F in (16, 128, 512):
+            out[f"c3_{opname}_F{F}"] = compact_resident_record(B, dataclasses.replace(c3, op=op, feat_dim=F), steps=20)
+    torch.cuda.empty_cache()
+    out["c5"] = c5_streamed_record(B, args)
+    return out
+
+
 def main():
     args = parse()
     w = gi.scaled(gi.WORKLOADS[args.workload], args.scale_down)
@@ -360,7 +593,8 @@ def main():
     gen_s = time.perf_counter() - t0
     K, F = w.hops, w.feat_dim
     F_total = F
-    if args.shard == "columns" and world > 1:
+    sharded = args.shard == "columns" and world > 1
+    if sharded:
         from paper_2207_12000_b200.shard import column_shard
         f_lo, f_hi = column_shard(F, world, rank)
         if f_hi == f_lo:
@@ -382,7 +616,7 @@ def main():
     if not args.ld and F % 4:
         args.ld = (F + 3) // 4 * 4  # the library wants leading dimensions that are multiples of 4 floats
     if args.ld:  # rows padded to the given leading dimension: strided views, the library takes ldx / ldo
-        assert args.ld >= F and args.ld % 4 == 0 and not (args.shard == "columns" and world > 1)
+        assert args.ld >= F and args.ld % 4 == 0 and not sharded
         Xp = torch.zeros((g.n, args.ld), dtype=torch.float32, device="cuda")
         Xp[:, :F] = X
         X = Xp[:, :F]
@@ -405,44 +639,10 @@ def main():
         with torch.cuda.graph(graph, stream=side):
             B.gnnpre_propagate(plan, X, K, outs, stream=side)
 
-    def step(want_stats, start=None):
-        if flush is not None:
-            flush.fill_(1)  # L2 flush between iterations, outside the timed interval
-        if start is not None:
-            start.record(stream)
-        if graph is not None and not want_stats:
-            graph.replay()  # on the current stream, the one the events are recorded on
-            return None
-        _, st = B.gnnpre_propagate(plan, X, K, outs, stream=stream, want_stats=want_stats)
-        return st
-
-    for _ in range(max(3, args.warmup)):
-        step(False)
-    barrier()
-
-    # ---------------- timed region: device-resident inputs, CUDA events on the launching stream.
-    # Pass 1 times exactly `steps` calls as a user makes them (asynchronous, no per-launch timers): `value`.
-    # Pass 2 repeats the same steps with the library's per-launch events on: the dominant kernel's duration.
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    seg_ms, seg_launches, launches = 0.0, 0, 0
-    with ClockSampler(local) as clocks:
-        barrier()
-        for a, b_ in ev:
-            step(False, start=a)
-            b_.record(stream)
-        barrier()
-        ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-        for a, b_ in ev2:
-            st = step(True, start=a)
-            b_.record(stream)
-            seg_ms += st.segments_ms
-            seg_launches += st.segments_launches
-            launches += st.kernel_launches
-        barrier()
-    step_ms = [a.elapsed_time(b_) for a, b_ in ev]
-    total_ms = float(sum(step_ms))
-    total_ms = max_over_ranks(total_ms, world, "cuda")
-    sharded = args.shard == "columns" and world > 1
+    # ---------------- timed region: device-resident inputs, CUDA events on the launching stream
+    t = time_resident(B, plan, X, K, outs, args.steps, args.warmup, flush, stream, graph=graph, barrier=barrier,
+                      sampler_index=local)
+    total_ms = max_over_ranks(t["total_ms"], world, "cuda")
     units_per_step = K * m * (F_total if sharded else F)
     # replicas: every rank does the whole workload; column shards: the ranks share one workload
     value = aggregate_throughput(units_per_step, args.steps, 1 if sharded else world, total_ms)
@@ -450,100 +650,85 @@ def main():
     # ---------------- roofline of the dominant kernel (the segment kernel: one launch = one hop here)
     peak, peak_kind = measured_peaks()
     gather_b, least_b = byte_model(g.n, m, F)
-    launches_per_hop = seg_launches / (args.steps * K)
-    seg_launch_ms = seg_ms / max(1, seg_launches)
-    achieved = gather_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9
-    traffic = (profiled_traffic(w.name) if args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1
-               and not args.no_bulk_copy and not args.feat_dim and args.op < 0 and not args.ld else None)
+    launches_per_hop = t["seg_launches"] / (args.steps * K)
+    seg_launch_ms = t["seg_ms"] / max(1, t["seg_launches"])
+    default_shape = (args.segment_edges == 0 and args.blocks < 0 and launches_per_hop == 1 and not args.no_bulk_copy
+                     and not args.feat_dim and args.op < 0 and not args.ld and args.scale_down == 1)
+    traffic = profiled_traffic(w.name) if default_shape else None
+    secs = seg_launch_ms * 1e-3
+    if traffic is not None:
+        achieved, basis = traffic / secs / 1e9, "DRAM bytes of one launch (ncu, dram__bytes_read.sum + dram__bytes_write.sum) / kernel time"
+        traffic_source = f"profiles/k_segments_tma_{w.name}_dram.md (ncu summary, kernel source hash matched)"
+    else:
+        achieved, basis = least_b / launches_per_hop / secs / 1e9, ("compulsory bytes of one launch (every matrix touched once: "
+                                                                   "8nF + 4|E| + 16n per hop) / kernel time; no ncu capture "
+                                                                   "matches these kernel sources and this workload")
+        traffic_source = None
+    ceil_ms = time_ceiling(B, plan, X, flush, stream) if world == 1 else None
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": traffic,
-                "dram_achieved": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9,
-                "dram_frac": None if traffic is None else traffic / (seg_launch_ms * 1e-3) / 1e9 / peak,
-                "model": "achieved = gather model: every neighbour row fetched once per edge, 4|E|F + 4nF + 4|E| + 16n "
-                         "bytes per hop; L2 hits make it exceed the DRAM peak; dram_achieved = ncu DRAM bytes / time",
-                "kernel": "k_segments", "kernel_ms_per_launch": seg_launch_ms,
+                "frac_basis": basis, "peak_kind": f"{peak_kind} copy bandwidth (burst)", "traffic": traffic,
+                "traffic_source": traffic_source,
+                "kernel": "k_segments_tma (bulk-copy segment kernel)" if 68 <= F <= 128 and not args.no_bulk_copy
+                          else "segment kernel (k_segments / k_segments_tma by tile width)",
+                "kernel_ms_per_launch": seg_launch_ms, "launches_per_hop": launches_per_hop,
                 "algorithmic_bytes_per_launch": gather_b / launches_per_hop,
-                "achieved_min_model": least_b / launches_per_hop / (seg_launch_ms * 1e-3) / 1e9,
+                "gather_model_gbs": gather_b / launches_per_hop / secs / 1e9,
+                "achieved_min_model": least_b / launches_per_hop / secs / 1e9,
+                "model": "algorithmic bytes = gather model, every neighbour row fetched once per edge: 4|E|F + 4nF + 4|E| + 16n "
+                         "per hop; L2 hits let gather_model_gbs exceed the DRAM peak, so frac is taken from DRAM traffic",
                 "kernel_timing": "second pass over the same steps with CUDA events around every launch of the kernel",
-                "kernel_share_of_step": seg_ms / sum(a.elapsed_time(b_) for a, b_ in ev2)}
+                "kernel_share_of_step": t["seg_ms"] / t["pass2_ms"],
+                "gather_ceiling_ms_per_hop": ceil_ms,
+                "frac_of_gather_ceiling": None if ceil_ms is None else ceil_ms / (seg_launch_ms * launches_per_hop)}
 
     # ---------------- end to end through the C ABI with host buffers (copies inside the timed region)
-    e2e = None
+    e2e, outs_h, Xh = None, None, None
     if not args.no_e2e and rank == 0:
         try:
-            Xh = torch.zeros((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F]
-            Xh.copy_(X)
-            outs_h = [torch.empty((g.n, ld), dtype=torch.float32, pin_memory=True)[:, :F] for _ in range(K)]
-            if w.streamed:  # the graph lives in pinned host memory too; its edge blocks are streamed
-                rp_e2e, ci_e2e = g.rowptr.cpu().pin_memory(), g.colidx.cpu().pin_memory()
-            else:
-                rp_e2e, ci_e2e = g.rowptr, g.colidx
-            hplan = B.gnnpre_build_plan(rp_e2e, ci_e2e, w.op, F, gin_eps=w.gin_eps, force_blocks=blocks,
-                                        force_col_slabs=args.e2e_col_slabs, segment_edges=args.segment_edges,
-                                        budget_bytes=int(args.budget_gb * 1e9), operands_mem=B.GNNPRE_MEM_HOST)
-            for _ in range(2):
-                B.gnnpre_propagate(hplan, Xh, K, outs_h)
-            reps = max(2, min(args.steps, 5))
-            torch.cuda.synchronize()
-            t0 = time.perf_counter()
-            for _ in range(reps):
-                _, hst = B.gnnpre_propagate(hplan, Xh, K, outs_h, want_stats=True)
-            torch.cuda.synchronize()
-            dt = (time.perf_counter() - t0) / reps
-            # column shards: rank 0 times its own slab through host buffers; the job's figure assumes the other
-            # ranks' slabs (same width but the last) take as long on their own host links
-            e2e_units = K * m * F * world if sharded else units_per_step
-            e2e = {"value": e2e_units / dt, "unit": UNIT, "h2d_bytes_per_step": int(hst.h2d_bytes),
-                   "d2h_bytes_per_step": int(hst.d2h_bytes), "ms_per_step": dt * 1e3,
-                   "col_slabs": hplan.info()["c"]}
-            hinfo = hplan.info()
-            e2e["blocks"] = hinfo["b"]
-            e2e["structure_on_host"] = bool(hinfo["structure_mem"])
+            e2e, outs_h, Xh = streamed_run(B, w, g, X, args, reps=max(2, min(args.steps, 5)), blocks=blocks,
+                                           col_slabs=args.e2e_col_slabs, ld=ld)
+            if sharded:  # rank 0 times its own slab; the job's figure assumes the other ranks' slabs take as long
+                e2e["value"] *= world
             # same bits are expected only when both plans cut the edge list the same way
-            comparable = hinfo["c"] == 1 and hinfo["b"] == info["b"] and hinfo["segment_edges"] == info["segment_edges"]
-            same = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if comparable else None
-            e2e["bitwise_equal_to_resident"] = same
+            comparable = e2e["blocks"] == info["b"] and e2e["segment_edges"] == info["segment_edges"] and F <= 128
+            e2e["bitwise_equal_to_resident"] = all(torch.equal(o.cpu(), h) for o, h in zip(outs, outs_h)) if comparable else None
             e2e["max_abs_diff_to_resident"] = max(float((o.cpu() - h).abs().max()) for o, h in zip(outs, outs_h))
-            hplan.close()
-            # host-link ceiling measured in this process: one 1 GiB pinned copy per direction, best of 3
-            pin = torch.empty(1 << 30, dtype=torch.uint8, pin_memory=True)
-            devb = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
-            link = {}
-            for name, dst, src in (("h2d_gbs", devb, pin), ("d2h_gbs", pin, devb)):
-                best = 0.0
-                for _ in range(3):
-                    torch.cuda.synchronize()
-                    t0 = time.perf_counter()
-                    dst.copy_(src, non_blocking=True)
-                    torch.cuda.synchronize()
-                    best = max(best, (1 << 30) / (time.perf_counter() - t0) / 1e9)
-                link[name] = best
-            moved = max(hst.h2d_bytes, hst.d2h_bytes)
-            link["achieved_gbs"] = moved / dt / 1e9
-            link["direction"] = "d2h" if hst.d2h_bytes >= hst.h2d_bytes else "h2d"
-            link["frac"] = link["achieved_gbs"] / link[link["direction"] + "_gbs"]
-            e2e["host_link"] = link
-            del pin, devb
         except B.GnnpreError as err:
             e2e = {"value": None, "unit": UNIT, "error": str(err)}
 
-    # ---------------- the oracle on this machine's host cores, bounded sample (rank 0, one GPU only)
+    # ---------------- the oracle on this machine's host cores, bounded sample (rank 0, one GPU only); the rows it
+    # computes are compared with hop 1 of the outputs that were timed
     cpu = None
     if not args.no_cpu_baseline and rank == 0 and world == 1:
-        cpu, _ = oracle_sample(w, g.to("cpu"), np.ascontiguousarray(X.cpu().numpy()), args.cpu_seconds)
+        got = {"resident": outs[0].cpu().numpy()}
+        if outs_h is not None:
+            got["host_buffers"] = outs_h[0].numpy()
+        cpu, _ = oracle_sample(w, g.to("cpu"), np.ascontiguousarray(X.cpu().numpy()), args.cpu_seconds, got=got)
+        if e2e is not None and "host_buffers" in cpu["parity"]:
+            e2e["parity_checked"] = bool(cpu["parity"]["host_buffers"]["ok"])
+    del outs_h, Xh
+
+    configs = None
+    if rank == 0 and world == 1 and args.workload == "c4" and default_shape and not args.no_configs:
+        plan.close()
+        del outs, X, flush
+        torch.cuda.empty_cache()
+        configs = configs_object(B, args)
 
     if rank == 0:
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(3, args.warmup), "ms_per_step": total_ms / args.steps, "higher_is_better": True,
                 "scaling": "strong" if sharded else "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-                "config": dict(workload_config(w, g, info), parallelism="column shards" if sharded else "replicas", cuda_graph=bool(args.cuda_graph), leading_dim=ld), "clocks": clocks.summary(), "e2e": e2e,
-                "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-                "plan_build_ms": plan_ms, "input_generation_s": gen_s,
+                "config": dict(workload_config(w, g, info), parallelism="column shards" if sharded else "replicas",
+                               cuda_graph=bool(args.cuda_graph), leading_dim=ld),
+                "clocks": t["clocks"], "e2e": e2e, "gpu_launches": int(t["launches"]), "roofline": roofline,
+                "cpu_baseline": cpu, "plan_build_ms": plan_ms, "input_generation_s": gen_s,
                 # the same metric if every step also rebuilt the plan (degrees, scales, Eq. 12, edge blocks, segments)
                 "value_including_plan_build": (1 if sharded else world) * units_per_step / ((total_ms / args.steps + plan_ms) * 1e-3),
-                "hop_ms": [float(st.hop_ms[k]) for k in range(K)]}
+                "hop_ms": t["hop_ms"], "configs": configs}
         print(json.dumps(line), flush=True)
-    plan.close()
+    if configs is None:
+        plan.close()
     if world > 1:
         dist.destroy_process_group()
 

@@ -129,7 +129,15 @@ typedef struct {
     int64_t h2d_bytes, d2h_bytes;  /* streamed runs */
     int64_t kernel_launches;       /* all kernels this call launched */
     int64_t segments_launches;     /* launches of the segment kernel among them */
+    float startup_ms;              /* streamed runs with host outputs: call start until the first output copy begins */
+    float drain_ms;                /* ... and from there until the last output copy has ended */
+    int32_t schedule;              /* GNNPRE_SCHEDULE_*: how the call was run */
+    int32_t upload_slabs;          /* column slabs X travelled in (streamed runs with host X) */
 } gnnpre_stats_t;
+
+#define GNNPRE_SCHEDULE_RESIDENT 0 /* everything on the device */
+#define GNNPRE_SCHEDULE_SLABS 1    /* Algorithm 1's loops, slab loop outermost: c equal slabs, each through all K hops */
+#define GNNPRE_SCHEDULE_PANELS 2   /* whole hop matrices on the device, narrow-first column panels (see gnnpre_propagate) */
 
 /*
  * Degrees D_i = number of nonzeros of row i (Section 2).  `deg_out` (int32[n]) lives in the same
@@ -179,6 +187,14 @@ int gnnpre_plan_support(const gnnpre_plan_t* plan, int64_t* rowptr_out, int32_t*
  * device->host on side streams while later blocks compute, and the call returns when out[] is
  * complete in host memory (GNNPRE_ERR_BUSY if another streamed call holds the plan).  Host buffers
  * should be page-locked for full link speed.
+ * Host X and host out[] together are run in one of two ways.  If the plan's budget has room for K + 1
+ * whole [n, F] matrices besides the plan, c was not forced, F >= 128 is a multiple of 32 and every host
+ * row starts on a 128-byte boundary, the hop matrices stay whole on the device and the columns travel in
+ * unequal slabs, narrow first (32, 32, 64, 128, ... columns, none wider than the plan's slab width): the
+ * first output rows can leave after 1/4 of the time an equal half of X would need, and later outputs
+ * leave in wide pieces (a departure from Algorithm 1's equal split ceil(d/c); every column is an
+ * independent product, so no result changes).  Otherwise Algorithm 1's loops run with the slab loop
+ * outermost, each of the c equal slabs of Eq. 12 through all K hops.  stats->schedule tells which.
  * Accumulation is fp32 in a fixed order: results are bitwise reproducible from run to run for a
  * given plan, and agree across different (b, c) or segment sizes only to rounding.
  * `stats` may be NULL; when given, device-resident calls synchronise `stream` to read the timers.
@@ -196,8 +212,10 @@ int gnnpre_propagate(gnnpre_plan_t* plan, const float* X, int64_t ldx, int32_t x
  * integer degrees and rounded once.  vals_out lives where vals_mem says.  Device-resident structure and
  * output: one launch on `stream`, asynchronous.  Otherwise the plan's b edge blocks play the role of
  * the paper's `a` passes - block E^(l) travels to the device if it lives on the host, its values travel
- * back if wanted on the host, two buffers taking turns - and the call returns when vals_out is complete
- * (GNNPRE_ERR_BUSY if a streamed call holds the plan).  gnnpre_propagate never needs this array.
+ * back if wanted on the host, on the plan's copy streams with two buffers of each kind taking turns, so
+ * that the upload of block l+1 and the download of block l-1 overlap the kernel of block l - and the call
+ * returns when vals_out is complete (GNNPRE_ERR_BUSY if a streamed call holds the plan).
+ * gnnpre_propagate never needs this array.
  */
 int gnnpre_normalize(gnnpre_plan_t* plan, float* vals_out, int32_t vals_mem, void* stream);
 
@@ -207,15 +225,42 @@ int gnnpre_solve_normalisation_blocks(int64_t B_A, int64_t B_S, int64_t B_D, int
                                       int64_t alpha_D, int64_t B_GPU, int64_t max_a, int64_t* a_out);
 
 /*
- * Failure-detection self-test (no counterpart in the paper).  The bulk-copy kernel never waits without
- * a limit: a wait that runs out sets an error word in the plan and the warp leaves; the next
- * synchronising call returns GNNPRE_ERR_TIMEOUT and clears the word.  This call exercises exactly that
- * path without any fault: one warp waits `polls` times (1..100000, each poll parks the warp for up to
- * 20 us) on a barrier that nothing completes.  Returns GNNPRE_ERR_TIMEOUT when the path works, and
- * leaves the device and the plan fully usable.  Synchronous.
+ * Whether a kernel of this plan gave up a wait (no counterpart in the paper).  The bulk-copy kernel never
+ * waits without a limit: a wait that runs out sets an error word in the plan, the warp leaves, and the rows
+ * it was working on are not valid.  Calls that synchronise anyway (streamed operands, or `stats` given)
+ * read that word themselves and return GNNPRE_ERR_TIMEOUT.  A device-resident call without `stats` only
+ * enqueues work and returns before it runs, so its caller asks here: this call synchronises `stream` (the
+ * stream the work was enqueued on), then returns GNNPRE_ERR_TIMEOUT if the word was set since it was last
+ * read, and clears it; GNNPRE_OK otherwise.  Call it after the last gnnpre_propagate /
+ * gnnpre_propagate_weighted of a batch, before trusting out[].
  */
+int gnnpre_plan_status(gnnpre_plan_t* plan, void* stream);
+
+/*
+ * Failure-detection self-test (no counterpart in the paper).  Exercises the give-up path described above
+ * without any fault: one warp waits `polls` times (1..100000, each poll parks the warp for up to 20 us) on
+ * a barrier that nothing completes, then sets the plan's error word and leaves.
+ *   gnnpre_selftest_wait_timeout_async  only enqueues that kernel on `stream`: the caller then sees
+ *                                       GNNPRE_ERR_TIMEOUT exactly once through gnnpre_plan_status
+ *   gnnpre_selftest_wait_timeout        enqueues it, synchronises and reads the word itself: returns
+ *                                       GNNPRE_ERR_TIMEOUT when the path works
+ * Either way the device and the plan stay fully usable.
+ */
+int gnnpre_selftest_wait_timeout_async(gnnpre_plan_t* plan, uint32_t polls, void* stream);
 int gnnpre_selftest_wait_timeout(gnnpre_plan_t* plan, uint32_t polls, void* stream);
 
+/*
+ * Failure injection for tests (no counterpart in the paper; nothing on the device is made to fail).  After
+ * this call the library's next `device_countdown` device allocations succeed and the one after them is
+ * reported as failed (GNNPRE_ERR_OOM_DEVICE) without calling the allocator; likewise `host_countdown`
+ * for page-locked host allocations (GNNPRE_ERR_OOM_HOST).  One failure per arming; a negative value
+ * disarms.  Process-wide.  A call that fails this way must leave no memory behind: gnnpre_build_plan
+ * returns *plan_out = NULL, a streamed gnnpre_propagate leaves the plan usable for the next call.
+ */
+int gnnpre_inject_alloc_failure(int64_t device_countdown, int64_t host_countdown);
+
+/* Waits for the plan's own streams and for the last device-resident call that used it (not for the whole
+ * device), then frees everything the plan owns. */
 void gnnpre_plan_destroy(gnnpre_plan_t* plan);
 
 /*
@@ -236,9 +281,15 @@ void gnnpre_plan_destroy(gnnpre_plan_t* plan);
  *   X, out     device, fp32 row-major [n, feat_dim] with leading dimensions ldx, ldo (multiples of 4,
  *              16-byte aligned bases, out != X); feat_dim a multiple of 4, at most 512
  * The work is enqueued on `stream`; the call returns at once and calls no cudaMalloc, cudaFree or
- * other allocating routine.  The first call on a device also looks up the device address of the
- * fixed array (once per device, with that device current), so make that first call outside any
- * stream capture.
+ * other allocating routine.
+ * First call on a device: it looks up the device address of the fixed array (once per device, with
+ * that device current).  With the driver's default lazy module loading that look-up is also the
+ * moment the part of the library that holds the array is loaded onto the device, i.e. when its
+ * GNNPRE_STATIC_SCRATCH_BYTES are reserved; if the device has no room left (a memory pool already
+ * owns all of it) that first call returns GNNPRE_ERR_OOM_DEVICE or GNNPRE_ERR_CUDA.  So make the first
+ * call at start-up, before the process freezes its footprint and outside any stream capture; later
+ * calls reserve nothing.  The address is cached per device for the life of the process and does not
+ * survive cudaDeviceReset: do not call this function again after resetting a device.
  * Limits: feat_dim <= 512 and 2 * ceil(nnz / 2^20) * feat_dim * 4 <= GNNPRE_STATIC_SCRATCH_BYTES,
  * else GNNPRE_ERR_TOO_LARGE (nothing is launched).
  * All calls on a device share the one array.  Each call overwrites the entries it later reads, so
@@ -327,6 +378,22 @@ int gnnpre_lc_first_layer(const float* const* hops, int32_t num_hops, int64_t n,
 int gnnpre_lc_selftest_wait_timeout(const float* hop, int64_t n, int64_t feat_dim, int64_t ldh, const float* Wt,
                                     int64_t hidden, int64_t ldw, float* Y, int64_t ldy, int32_t* error_flag,
                                     uint32_t polls, void* stream);
+
+/*
+ * Measurement aid (no counterpart in the paper): the fetches of ONE hop and nothing else.  Walks the plan's
+ * segments exactly as gnnpre_propagate's segment kernels do - same column tiles, same index stream, same
+ * fetch path (128-bit loads into registers, or bulk copies into shared memory, by row width) - adds every
+ * fetched row into a plain running sum and writes one float per segment to `sink`.  No scales, no row ends,
+ * no compensated sums, no output rows.  Its duration is the yardstick for matrices that fit the L2, where
+ * the HBM roofline does not bound a hop: segment-kernel time / this time is the fraction of the device's own
+ * gather speed that the kernel reaches.
+ *   plan    device-resident structure (else INVALID_ARG)
+ *   X       device fp32 [n, F], leading dimension ldx (multiple of 4, base 16-byte aligned)
+ *   sink    device fp32 [num_segments] (gnnpre_plan_info); contents meaningless
+ * Enqueued on `stream`, asynchronous; the caller times it.  A bounded wait that runs out is reported through
+ * gnnpre_plan_status like any other.
+ */
+int gnnpre_gather_ceiling(gnnpre_plan_t* plan, const float* X, int64_t ldx, float* sink, void* stream);
 
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;

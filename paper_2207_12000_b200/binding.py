@@ -18,6 +18,7 @@ GNNPRE_OP_GCN_SYM, GNNPRE_OP_SAGE_MEAN, GNNPRE_OP_GIN_SUM = 0, 1, 2
 GNNPRE_MEM_DEVICE, GNNPRE_MEM_HOST = 0, 1
 GNNPRE_FLAG_LAUNCH_PER_BLOCK, GNNPRE_FLAG_SKIP_VALIDATION, GNNPRE_FLAG_NO_BULK_COPY = 1, 2, 4
 GNNPRE_MAX_HOPS = 64
+GNNPRE_SCHEDULE_RESIDENT, GNNPRE_SCHEDULE_SLABS, GNNPRE_SCHEDULE_PANELS = 0, 1, 2
 
 
 class gnnpre_csr_t(ctypes.Structure):
@@ -56,7 +57,9 @@ class gnnpre_block_info_t(ctypes.Structure):
 class gnnpre_stats_t(ctypes.Structure):
     _fields_ = [("hop_ms", ctypes.c_float * GNNPRE_MAX_HOPS), ("total_ms", ctypes.c_float),
                 ("segments_ms", ctypes.c_float), ("h2d_bytes", ctypes.c_int64), ("d2h_bytes", ctypes.c_int64),
-                ("kernel_launches", ctypes.c_int64), ("segments_launches", ctypes.c_int64)]
+                ("kernel_launches", ctypes.c_int64), ("segments_launches", ctypes.c_int64),
+                ("startup_ms", ctypes.c_float), ("drain_ms", ctypes.c_float), ("schedule", ctypes.c_int32),
+                ("upload_slabs", ctypes.c_int32)]
 
 
 class GnnpreError(RuntimeError):
@@ -92,6 +95,10 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_normalize.argtypes = [p, p, i32, p]
     lib.gnnpre_solve_normalisation_blocks.argtypes = [i64] * 8 + [ctypes.POINTER(i64)]
     lib.gnnpre_selftest_wait_timeout.argtypes = [p, ctypes.c_uint32, p]
+    lib.gnnpre_selftest_wait_timeout_async.argtypes = [p, ctypes.c_uint32, p]
+    lib.gnnpre_plan_status.argtypes = [p, p]
+    lib.gnnpre_gather_ceiling.argtypes = [p, p, i64, p, p]
+    lib.gnnpre_inject_alloc_failure.argtypes = [i64, i64]
     lib.gnnpre_plan_destroy.argtypes = [p]
     lib.gnnpre_plan_destroy.restype = None
     lib.gnnpre_solve_budget.argtypes = [i64] * 8 + [ctypes.POINTER(i64), ctypes.POINTER(i64)]
@@ -344,6 +351,35 @@ def gnnpre_selftest_wait_timeout(plan: Plan, polls: int = 200, stream=None) -> i
     return int(_lib.gnnpre_selftest_wait_timeout(plan.handle, polls, _stream_ptr(stream)))
 
 
+def gnnpre_selftest_wait_timeout_async(plan: Plan, polls: int = 200, stream=None) -> None:
+    """Enqueues the wait that runs out; gnnpre_plan_status then reports it once."""
+    _check(_lib.gnnpre_selftest_wait_timeout_async(plan.handle, polls, _stream_ptr(stream)),
+           "gnnpre_selftest_wait_timeout_async")
+
+
+def gnnpre_plan_status(plan: Plan, stream=None) -> int:
+    """Synchronises `stream` and returns 0, or -8 (GNNPRE_ERR_TIMEOUT) once if a kernel of the plan gave up a wait."""
+    return int(_lib.gnnpre_plan_status(plan.handle, _stream_ptr(stream)))
+
+
+def gnnpre_gather_ceiling(plan: Plan, X: torch.Tensor, sink: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """Enqueues the fetches of one hop (rows summed plainly, nothing stored but one float per segment): the
+    yardstick the segment kernels are measured against when X fits the L2.  Returns the sink buffer."""
+    assert X.is_cuda and X.dtype == torch.float32 and X.dim() == 2 and X.stride(1) == 1
+    nseg = gnnpre_plan_info(plan)["num_segments"]
+    if sink is None:
+        sink = torch.empty(max(nseg, 1), dtype=torch.float32, device=X.device)
+    assert sink.is_cuda and sink.dtype == torch.float32 and sink.numel() >= nseg and sink.is_contiguous()
+    _check(_lib.gnnpre_gather_ceiling(plan.handle, X.data_ptr(), X.stride(0), sink.data_ptr(), _stream_ptr(stream)),
+           "gnnpre_gather_ceiling")
+    return sink
+
+
+def gnnpre_inject_alloc_failure(device_countdown: int = -1, host_countdown: int = -1) -> None:
+    """Test hook: the library's (countdown + 1)-th next allocation of that kind is reported as failed; -1 disarms."""
+    _check(_lib.gnnpre_inject_alloc_failure(device_countdown, host_countdown), "gnnpre_inject_alloc_failure")
+
+
 def gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c):
     b, c = ctypes.c_int64(), ctypes.c_int64()
     rc = _lib.gnnpre_solve_budget(B_S, B_X, B_fixed, beta_S, beta_X, B_GPU, max_b, max_c, ctypes.byref(b),
@@ -361,5 +397,6 @@ def gnnpre_status_string(status: int) -> str:
 def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
             "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_propagate_weighted", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_lc_selftest_wait_timeout", "gnnpre_normalize",
-            "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_selftest_wait_timeout_async",
+            "gnnpre_plan_status", "gnnpre_inject_alloc_failure", "gnnpre_gather_ceiling", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

@@ -1,4 +1,5 @@
 // C-ABI glue: argument checks, status text, and the dispatch of gnnpre_propagate.
+#include <atomic>
 #include <cstdio>
 #include <cstring>
 
@@ -8,6 +9,35 @@ namespace gnnpre {
 
 namespace {
 thread_local char g_last_error[512] = "";
+// Allocations still allowed to succeed before one is reported as failed; negative = no injection.
+std::atomic<int64_t> g_fail_countdown[2] = {{-1}, {-1}};
+
+// Whether the [n, width] matrices at a (leading dimension lda floats) and b (ldb) share an element.  Column
+// views of one wider buffer (equal leading dimensions, disjoint column ranges) do not.
+bool matrices_overlap(const float* a, int64_t lda, const float* b, int64_t ldb, int64_t n, int64_t width) {
+    if (n < 1 || width < 1) return false;
+    const intptr_t pa = reinterpret_cast<intptr_t>(a), pb = reinterpret_cast<intptr_t>(b);
+    const intptr_t span_a = ((n - 1) * lda + width) * (intptr_t)sizeof(float);
+    const intptr_t span_b = ((n - 1) * ldb + width) * (intptr_t)sizeof(float);
+    if (pa + span_a <= pb || pb + span_b <= pa) return false;  // the address ranges are disjoint
+    if (lda != ldb) return true;                                // interleaved with different strides: assume they touch
+    // same stride: element (i, p) of a meets (j, q) of b iff d = (i - j) * ld + (p - q), |p - q| < width
+    const intptr_t diff = pb - pa;
+    if (diff % (intptr_t)sizeof(float) != 0) return true;
+    const intptr_t d = diff / (intptr_t)sizeof(float);
+    intptr_t r = d % lda;
+    if (r < 0) r += lda;
+    return r < width || r > lda - width;
+}
+}  // namespace
+
+bool injected_alloc_failure(int kind) {
+    std::atomic<int64_t>& c = g_fail_countdown[kind];
+    int64_t v = c.load();
+    while (v >= 0) {
+        if (c.compare_exchange_weak(v, v - 1)) return v == 0;  // the allocation that finds 0 fails; -1 = disarmed
+    }
+    return false;
 }
 
 void set_last_cuda_error(cudaError_t e, const char* what, const char* file, int line) {
@@ -51,9 +81,10 @@ extern "C" int gnnpre_propagate(gnnpre_plan_t* P, const float* X, int64_t ldx, i
     for (int32_t k = 0; k < K; ++k) {
         if (!out[k]) return GNNPRE_ERR_INVALID_ARG;
         if (reinterpret_cast<uintptr_t>(out[k]) & 15u) return GNNPRE_ERR_ALIGN;
-        if (out[k] == X) return GNNPRE_ERR_INVALID_ARG;
+        // host and device addresses live in one address space (unified addressing), so one test serves both
+        if (matrices_overlap(X, ldx, out[k], ldo, P->n, P->feat_dim)) return GNNPRE_ERR_INVALID_ARG;
         for (int32_t j = 0; j < k; ++j)
-            if (out[j] == out[k]) return GNNPRE_ERR_INVALID_ARG;
+            if (matrices_overlap(out[j], ldo, out[k], ldo, P->n, P->feat_dim)) return GNNPRE_ERR_INVALID_ARG;
     }
     if (stats) std::memset(stats, 0, sizeof(*stats));
     int dev = -1;
@@ -72,17 +103,33 @@ extern "C" int gnnpre_propagate_weighted(gnnpre_plan_t* P, const float* X, int64
     if (ldx < P->feat_dim || ldo < P->feat_dim || ldz < P->feat_dim) return GNNPRE_ERR_INVALID_ARG;
     if (ldx % 4 != 0 || ldo % 4 != 0 || ldz % 4 != 0) return GNNPRE_ERR_ALIGN;
     if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(Z) & 15u)) return GNNPRE_ERR_ALIGN;
-    if (Z == X) return GNNPRE_ERR_INVALID_ARG;
+    if (matrices_overlap(X, ldx, Z, ldz, P->n, P->feat_dim)) return GNNPRE_ERR_INVALID_ARG;
     for (int32_t k = 0; k < K; ++k) {
-        if (!out[k] || out[k] == X || out[k] == Z) return GNNPRE_ERR_INVALID_ARG;
+        if (!out[k]) return GNNPRE_ERR_INVALID_ARG;
         if (reinterpret_cast<uintptr_t>(out[k]) & 15u) return GNNPRE_ERR_ALIGN;
+        if (matrices_overlap(X, ldx, out[k], ldo, P->n, P->feat_dim) ||
+            matrices_overlap(Z, ldz, out[k], ldo, P->n, P->feat_dim))
+            return GNNPRE_ERR_INVALID_ARG;
         // a hop may reuse the buffer of the hop before the previous one (two buffers suffice when only Z is wanted),
         // but never the one it reads
-        if (k > 0 && out[k] == out[k - 1]) return GNNPRE_ERR_INVALID_ARG;
+        if (k > 0 && matrices_overlap(out[k - 1], ldo, out[k], ldo, P->n, P->feat_dim)) return GNNPRE_ERR_INVALID_ARG;
     }
     int dev = -1;
     GNNPRE_CUDA(cudaGetDevice(&dev));
     if (dev != P->device) return GNNPRE_ERR_INVALID_ARG;
     WeightedSum w{gamma, Z, ldz};
     return propagate_resident(P, X, ldx, K, out, ldo, static_cast<cudaStream_t>(stream), nullptr, &w);
+}
+
+// See include/gnnpre.h.
+extern "C" int gnnpre_plan_status(gnnpre_plan_t* P, void* stream) {
+    if (!P) return GNNPRE_ERR_INVALID_ARG;
+    GNNPRE_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(stream)));
+    return check_device_error(P);
+}
+
+extern "C" int gnnpre_inject_alloc_failure(int64_t device_countdown, int64_t host_countdown) {
+    g_fail_countdown[0].store(device_countdown < 0 ? -1 : device_countdown);
+    g_fail_countdown[1].store(host_countdown < 0 ? -1 : host_countdown);
+    return GNNPRE_OK;
 }

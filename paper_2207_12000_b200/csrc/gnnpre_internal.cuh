@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units.
 #pragma once
 
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -29,6 +30,10 @@ void set_last_cuda_error(cudaError_t e, const char* what, const char* file, int 
         if (s__ != GNNPRE_OK) return s__; \
     } while (0)
 
+// Failure injection for tests (gnnpre_inject_alloc_failure): true when this allocation must be
+// reported as failed.  kind 0 = device memory, 1 = page-locked host memory.
+bool injected_alloc_failure(int kind);
+
 // Device allocation that frees itself.
 template <typename T>
 struct DevBuf {
@@ -46,6 +51,10 @@ struct DevBuf {
     int alloc(size_t n) {
         reset();
         if (n == 0) return GNNPRE_OK;
+        if (injected_alloc_failure(0)) {
+            set_last_cuda_error(cudaErrorMemoryAllocation, "cudaMalloc (injected failure)", __FILE__, __LINE__);
+            return GNNPRE_ERR_OOM_DEVICE;
+        }
         GNNPRE_CUDA(cudaMalloc(reinterpret_cast<void**>(&p), n * sizeof(T)));
         count = n;
         return GNNPRE_OK;
@@ -70,7 +79,8 @@ struct PinnedBuf {
     int alloc(size_t n) {
         reset();
         if (n == 0) return GNNPRE_OK;
-        cudaError_t e = cudaMallocHost(reinterpret_cast<void**>(&p), n * sizeof(T));
+        cudaError_t e = injected_alloc_failure(1) ? cudaErrorMemoryAllocation
+                                                  : cudaMallocHost(reinterpret_cast<void**>(&p), n * sizeof(T));
         if (e != cudaSuccess) {
             set_last_cuda_error(e, "cudaMallocHost", __FILE__, __LINE__);
             (void)cudaGetLastError();
@@ -102,12 +112,14 @@ struct Segment {
 };
 
 // A row whose edges span segments seg_first..seg_last: its result is
-// rscale[row] * (tail part of seg_first + head parts of seg_first+1 .. seg_last).
+// rscale[row] * (tail part of seg_first + head parts of seg_first+1 .. seg_last).  Those parts lie in
+// consecutive scratch rows slot0, slot0 + 1, ... (the segments between the first and the last lie wholly
+// inside the row, so each owns exactly one slot, and slots are numbered in segment order).
 struct RowFixup {
     int32_t row;
     int32_t seg_first;
     int32_t seg_last;
-    int32_t pad;
+    int32_t slot0;
 };
 
 struct Block {
@@ -116,6 +128,7 @@ struct Block {
     int32_t first_partial, last_partial;
     int64_t seg_lo, seg_hi;            // segments of this block
     int64_t fix_lo, fix_hi;            // fix-ups whose last segment lies in this block
+    int64_t hub_lo, hub_hi;            // those among them with more than hub_parts parts (entries of `hubs`)
     int64_t done_row_lo, done_row_hi;  // rows complete once this block has run: [lo, hi)
 };
 
@@ -151,14 +164,30 @@ struct gnnpre_plan {
     std::vector<gnnpre::Block> blocks;
     gnnpre::DevBuf<gnnpre::Segment> segments;  // num_segments + 1 (the sentinel carries the end edge)
     gnnpre::DevBuf<gnnpre::RowFixup> fixups;
+    gnnpre::DevBuf<int32_t> hubs;      // indices of the fix-ups with more than hub_parts parts, ascending
+    int64_t num_hubs = 0;
+    int32_t hub_parts = 0;
     int64_t num_segments = 0, num_fixups = 0, num_slots = 0;
     gnnpre::DevBuf<float> scratch;  // num_slots rows of slab_width floats
     gnnpre::DevBuf<int> dev_error;  // set by a kernel whose bounded wait ran out
     int num_sms = 0;
+    // tensor maps of the matrices the bulk-copy kernel has been launched on (a cache: not part of the plan's meaning)
+    struct TensorMapEntry {
+        const float* x;
+        int64_t ldx;
+        int32_t f4;
+        CUtensorMap map;
+    };
+    mutable std::vector<TensorMapEntry> tmaps;
     // streaming state
     gnnpre::DevBuf<float> slab[4];
-    cudaStream_t s_h2d = nullptr, s_d2h = nullptr, s_compute = nullptr;
+    std::vector<gnnpre::DevBuf<float>> whole;  // panel schedule: X_0 .. X_K, each [n, feat_dim], grown on demand
+    bool col_slabs_forced = false;             // c was given by the caller: the slab loop is then kept as asked
+    cudaStream_t s_h2d = nullptr, s_d2h = nullptr, s_compute = nullptr, s_struct = nullptr;
     int busy = 0;
+    // recorded on the caller's stream after the last work of every device-resident call: what
+    // gnnpre_plan_destroy waits for instead of the whole device
+    cudaEvent_t last_use = nullptr;
 
     ~gnnpre_plan();
     int64_t device_bytes() const;
@@ -188,7 +217,8 @@ struct HopArgs {
 
 // propagate.cu
 int launch_segments(const gnnpre_plan* plan, const HopArgs& a, int64_t seg_lo, int64_t seg_hi, cudaStream_t stream);
-int launch_fixups(const gnnpre_plan* plan, const HopArgs& a, int64_t fix_lo, int64_t fix_hi, cudaStream_t stream);
+int launch_fixups(const gnnpre_plan* plan, const HopArgs& a, int64_t fix_lo, int64_t fix_hi, int64_t hub_lo, int64_t hub_hi,
+                  cudaStream_t stream);
 int launch_zero_empty_rows(const gnnpre_plan* plan, const HopArgs& a, cudaStream_t stream);
 struct WeightedSum {         // optional extra output of propagate_resident
     const float* gamma;      // host, K + 1 weights
@@ -199,6 +229,7 @@ int propagate_resident(gnnpre_plan* plan, const float* X, int64_t ldx, int32_t K
                        cudaStream_t stream, gnnpre_stats_t* stats, const WeightedSum* wsum = nullptr);
 
 // stream.cu
+int ensure_streams(gnnpre_plan* plan);  // creates the plan's three side streams on first use
 int propagate_streamed(gnnpre_plan* plan, const float* X, int64_t ldx, int32_t x_mem, int32_t K, float* const* out,
                        int64_t ldo, int32_t out_mem, cudaStream_t stream, gnnpre_stats_t* stats);
 

@@ -3,6 +3,7 @@
 // applies the per-node scales on the fly); this export serves callers that want S as a matrix.
 // Every value is evaluated in fp64 from the integer degrees and rounded once to fp32.
 #include <algorithm>
+#include <vector>
 
 #include "gnnpre_internal.cuh"
 
@@ -82,57 +83,92 @@ extern "C" int gnnpre_normalize(gnnpre_plan_t* P, float* vals_out, int32_t vals_
         a.out_base = 0;
         return launch_values(a, st);
     }
-    // Block by block (the paper's a passes): E^(l) up if it lives on the host, values of block l down if
-    // the caller wants them on the host, two buffers of each taking turns so copies and kernels overlap.
+    // Block by block (the paper's a passes): E^(l) goes up on the plan's upload stream if it lives on the
+    // host, the kernel runs on its compute stream, the values of block l go down on its download stream if
+    // the caller wants them on the host.  Two buffers of each kind take turns and events order the three
+    // streams, so block l+1 uploads and block l-1 downloads while block l computes.
     if (__sync_lock_test_and_set(&P->busy, 1)) return GNNPRE_ERR_BUSY;
     int64_t longest = 0;
     for (const Block& B : P->blocks) longest = std::max(longest, B.e_hi - B.e_lo);
     DevBuf<float> stage[2];
-    int rc = GNNPRE_OK;
-    if (vals_mem == GNNPRE_MEM_HOST) {
-        rc = stage[0].alloc((size_t)longest);
-        if (rc == GNNPRE_OK && P->blocks.size() > 1) rc = stage[1].alloc((size_t)longest);
-    }
-    for (size_t j = 0; j < P->blocks.size() && rc == GNNPRE_OK; ++j) {
-        const Block& B = P->blocks[j];
-        const int sb = (int)(j & 1);
-        a.row_lo = B.row_lo;
-        a.row_hi = B.row_hi;
-        a.e_lo = B.e_lo;
-        a.e_hi = B.e_hi;
-        cudaError_t e = cudaSuccess;
-        if (e_host) {
-            // same-stream order keeps the staging buffers safe: block j+2's upload follows block j's kernel
-            if (P->stage_holds[sb] != (int64_t)j) {
-                e = cudaMemcpyAsync(P->colx_stage[sb].p, P->colx_host.p + B.e_lo, sizeof(uint32_t) * (size_t)(B.e_hi - B.e_lo),
-                                    cudaMemcpyHostToDevice, st);
-                P->stage_holds[sb] = (int64_t)j;
-            }
-            a.colx = P->colx_stage[sb].p;
-            a.colx_base = B.e_lo;
-        } else {
-            a.colx = P->colx.p;
-            a.colx_base = 0;
-        }
+    std::vector<cudaEvent_t> events;
+    auto record = [&](cudaStream_t s, cudaEvent_t* out) -> int {
+        cudaEvent_t e = nullptr;
+        GNNPRE_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        events.push_back(e);
+        GNNPRE_CUDA(cudaEventRecord(e, s));
+        *out = e;
+        return GNNPRE_OK;
+    };
+    auto wait = [&](cudaStream_t s, cudaEvent_t e) -> int {
+        if (e) GNNPRE_CUDA(cudaStreamWaitEvent(s, e, 0));
+        return GNNPRE_OK;
+    };
+    auto body = [&]() -> int {
+        GNNPRE_TRY(ensure_streams(P));
         if (vals_mem == GNNPRE_MEM_HOST) {
-            a.out = stage[sb].p;
-            a.out_base = B.e_lo;
-        } else {
-            a.out = vals_out;
-            a.out_base = 0;
+            GNNPRE_TRY(stage[0].alloc((size_t)longest));
+            if (P->blocks.size() > 1) GNNPRE_TRY(stage[1].alloc((size_t)longest));
         }
-        if (e == cudaSuccess) rc = launch_values(a, st);
-        if (e == cudaSuccess && rc == GNNPRE_OK && vals_mem == GNNPRE_MEM_HOST)
-            e = cudaMemcpyAsync(vals_out + B.e_lo, stage[sb].p, sizeof(float) * (size_t)(B.e_hi - B.e_lo),
-                                cudaMemcpyDeviceToHost, st);
-        if (e != cudaSuccess) {
-            set_last_cuda_error(e, "gnnpre_normalize copy", __FILE__, __LINE__);
-            rc = GNNPRE_ERR_CUDA;
+        cudaEvent_t start = nullptr;
+        GNNPRE_TRY(record(st, &start));
+        GNNPRE_TRY(wait(P->s_h2d, start));
+        GNNPRE_TRY(wait(P->s_compute, start));
+        GNNPRE_TRY(wait(P->s_d2h, start));
+        cudaEvent_t kernel_done[2] = {nullptr, nullptr};  // last kernel that read edge buffer sb / wrote value buffer sb
+        cudaEvent_t drained[2] = {nullptr, nullptr};      // last download out of value buffer sb
+        for (size_t j = 0; j < P->blocks.size(); ++j) {
+            const Block& B = P->blocks[j];
+            const int sb = (int)(j & 1);
+            a.row_lo = B.row_lo;
+            a.row_hi = B.row_hi;
+            a.e_lo = B.e_lo;
+            a.e_hi = B.e_hi;
+            if (e_host) {
+                if (P->stage_holds[sb] != (int64_t)j) {
+                    GNNPRE_TRY(wait(P->s_h2d, kernel_done[sb]));
+                    GNNPRE_CUDA(cudaMemcpyAsync(P->colx_stage[sb].p, P->colx_host.p + B.e_lo,
+                                                sizeof(uint32_t) * (size_t)(B.e_hi - B.e_lo), cudaMemcpyHostToDevice,
+                                                P->s_h2d));
+                    P->stage_holds[sb] = (int64_t)j;
+                    cudaEvent_t up = nullptr;
+                    GNNPRE_TRY(record(P->s_h2d, &up));
+                    GNNPRE_TRY(wait(P->s_compute, up));
+                }
+                a.colx = P->colx_stage[sb].p;
+                a.colx_base = B.e_lo;
+            } else {
+                a.colx = P->colx.p;
+                a.colx_base = 0;
+            }
+            if (vals_mem == GNNPRE_MEM_HOST) {
+                GNNPRE_TRY(wait(P->s_compute, drained[sb]));
+                a.out = stage[sb].p;
+                a.out_base = B.e_lo;
+            } else {
+                a.out = vals_out;
+                a.out_base = 0;
+            }
+            GNNPRE_TRY(launch_values(a, P->s_compute));
+            GNNPRE_TRY(record(P->s_compute, &kernel_done[sb]));
+            if (vals_mem == GNNPRE_MEM_HOST) {
+                GNNPRE_TRY(wait(P->s_d2h, kernel_done[sb]));
+                GNNPRE_CUDA(cudaMemcpyAsync(vals_out + B.e_lo, stage[sb].p, sizeof(float) * (size_t)(B.e_hi - B.e_lo),
+                                            cudaMemcpyDeviceToHost, P->s_d2h));
+                GNNPRE_TRY(record(P->s_d2h, &drained[sb]));
+            }
         }
-    }
+        return GNNPRE_OK;
+    };
+    int rc = body();
     // the staging buffers die with this call, and host results are promised on return
-    if (cudaStreamSynchronize(st) != cudaSuccess && rc == GNNPRE_OK) rc = GNNPRE_ERR_CUDA;
-    if (rc != GNNPRE_OK) P->stage_holds[0] = P->stage_holds[1] = -1;
+    for (cudaStream_t s : {P->s_h2d, P->s_compute, P->s_d2h})
+        if (s && cudaStreamSynchronize(s) != cudaSuccess && rc == GNNPRE_OK) rc = GNNPRE_ERR_CUDA;
+    for (cudaEvent_t e : events) cudaEventDestroy(e);
+    if (rc != GNNPRE_OK) {
+        (void)cudaGetLastError();
+        P->stage_holds[0] = P->stage_holds[1] = -1;
+    }
     __sync_lock_release(&P->busy);
     return rc;
 }

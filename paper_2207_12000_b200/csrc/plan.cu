@@ -319,11 +319,30 @@ __global__ void k_segment_finalize(int64_t nseg, Segment* __restrict__ segs, con
         f.row = row;
         f.seg_first = (int32_t)lo;
         f.seg_last = (int32_t)s;
-        f.pad = 0;
+        f.slot0 = slot_scan[2 * lo + 1];  // the tail slot of the row's first segment; the other parts follow it
         fixups[emit_scan[s]] = f;
     }
     segs[s].slot_head = flags[2 * s] ? slot_scan[2 * s] : -1;
     segs[s].slot_tail = flags[2 * s + 1] ? slot_scan[2 * s + 1] : -1;
+}
+
+__global__ void k_hub_flags(int64_t nfix, const RowFixup* __restrict__ fix, int32_t hub_parts, int32_t* __restrict__ flag) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nfix) flag[i] = fix[i].seg_last - fix[i].seg_first + 1 > hub_parts;
+}
+
+__global__ void k_hub_scatter(int64_t nfix, const int32_t* __restrict__ flag, const int32_t* __restrict__ scan,
+                              int32_t* __restrict__ hubs) {
+    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < nfix && flag[i]) hubs[scan[i]] = (int32_t)i;
+}
+
+// Parts beyond which a cut row counts as a hub and gets a whole CTA of the fix-up kernel (64 chains) instead of a
+// warp (8 chains).  One value for all widths up to 128 columns, because the tree's shape decides the bits and
+// those must not depend on how a matrix is cut into column tiles; wider tiles hold fewer parts per batch of loads.
+int32_t hub_parts_for(int64_t width) {
+    const int64_t f4 = std::min<int64_t>(std::max<int64_t>(width, 4), 512) / 4;
+    return f4 <= 32 ? 64 : f4 <= 64 ? 32 : 16;
 }
 
 __global__ void k_clear_pad(int64_t nseg, Segment* __restrict__ segs) {
@@ -419,13 +438,16 @@ gnnpre_plan::~gnnpre_plan() {
     if (s_h2d) cudaStreamDestroy(s_h2d);
     if (s_d2h) cudaStreamDestroy(s_d2h);
     if (s_compute) cudaStreamDestroy(s_compute);
+    if (s_struct) cudaStreamDestroy(s_struct);
+    if (last_use) cudaEventDestroy(last_use);
 }
 
 int64_t gnnpre_plan::device_bytes() const {
     size_t t = deg.bytes() + rscale.bytes() + cscale.bytes() + nzrows.bytes() + emptyrows.bytes() + rowptr_t.bytes() +
-               colx.bytes() + colx_stage[0].bytes() + colx_stage[1].bytes() + segments.bytes() + fixups.bytes() +
+               colx.bytes() + colx_stage[0].bytes() + colx_stage[1].bytes() + segments.bytes() + fixups.bytes() + hubs.bytes() +
                scratch.bytes() + dev_error.bytes();
     for (const auto& s : slab) t += s.bytes();
+    for (const auto& s : whole) t += s.bytes();
     return (int64_t)t;
 }
 
@@ -557,6 +579,7 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     const int64_t max_b = std::min<int64_t>(std::max<int64_t>(m, 1), 1 << 20);
     int64_t b = opts->force_blocks, c = opts->force_col_slabs;
     if (b < 0 || c < 0 || c > max_c) return GNNPRE_ERR_INVALID_ARG;
+    P->col_slabs_forced = c > 0;
     if (b > 0 && b > m) return GNNPRE_ERR_INVALID_ARG;
     if (b == 0 || c == 0) {
         // a forced value pins that variable; the other is searched
@@ -631,7 +654,7 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     GNNPRE_TRY(P->segments.alloc((size_t)nseg + 1));
     if (m == 0) {
         // no edges at all: every row is empty; one empty block
-        P->blocks[0] = Block{0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, n};
+        P->blocks[0] = Block{0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, 0, n};
         Segment sentinel{0, 0, -1, -1, 0};
         GNNPRE_CUDA(cudaMemcpy(P->segments.p, &sentinel, sizeof(Segment), cudaMemcpyHostToDevice));
         return GNNPRE_OK;
@@ -683,6 +706,35 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     std::vector<int32_t> fix_at((size_t)b + 1);
     GNNPRE_CUDA(cudaMemcpy(fix_at.data(), d_fix_at.p, sizeof(int32_t) * (size_t)(b + 1), cudaMemcpyDeviceToHost));
 
+    // hub rows (more parts than a warp adds quickly) are listed so that the fix-up kernel can give each a CTA
+    P->hub_parts = hub_parts_for(P->slab_width);
+    std::vector<int32_t> hub_at((size_t)b + 1, 0);
+    if (n_fix > 0) {
+        DevBuf<int32_t> hub_flag, hub_scan, d_hub_at;
+        DevBuf<int64_t> d_fix_at64;
+        GNNPRE_TRY(hub_flag.alloc((size_t)n_fix));
+        GNNPRE_TRY(hub_scan.alloc((size_t)n_fix + 1));
+        k_hub_flags<<<grid_for(n_fix, kTB), kTB, 0, st>>>(n_fix, P->fixups.p, P->hub_parts, hub_flag.p);
+        GNNPRE_CUDA(cudaGetLastError());
+        GNNPRE_TRY(exclusive_scan(hub_flag.p, n_fix, hub_scan.p, st));
+        int32_t n_hubs = 0;
+        GNNPRE_CUDA(cudaMemcpy(&n_hubs, hub_scan.p + n_fix, sizeof(int32_t), cudaMemcpyDeviceToHost));
+        P->num_hubs = n_hubs;
+        if (n_hubs > 0) {
+            GNNPRE_TRY(P->hubs.alloc((size_t)n_hubs));
+            k_hub_scatter<<<grid_for(n_fix, kTB), kTB, 0, st>>>(n_fix, hub_flag.p, hub_scan.p, P->hubs.p);
+            GNNPRE_CUDA(cudaGetLastError());
+            std::vector<int64_t> fix_at64(fix_at.begin(), fix_at.end());
+            GNNPRE_TRY(d_fix_at64.alloc((size_t)b + 1));
+            GNNPRE_TRY(d_hub_at.alloc((size_t)b + 1));
+            GNNPRE_CUDA(cudaMemcpy(d_fix_at64.p, fix_at64.data(), sizeof(int64_t) * (size_t)(b + 1), cudaMemcpyHostToDevice));
+            k_gather_i32<<<grid_for(b + 1, kTB), kTB, 0, st>>>((int)(b + 1), d_fix_at64.p, hub_scan.p, d_hub_at.p);
+            GNNPRE_CUDA(cudaGetLastError());
+            GNNPRE_CUDA(cudaMemcpy(hub_at.data(), d_hub_at.p, sizeof(int32_t) * (size_t)(b + 1), cudaMemcpyDeviceToHost));
+        }
+        GNNPRE_CUDA(cudaStreamSynchronize(st));  // temporaries die here
+    }
+
     for (int64_t l = 0; l < b; ++l) {
         Block& B = P->blocks[(size_t)l];
         const BlockRows& r = h_rows[(size_t)l];
@@ -696,6 +748,8 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
         B.seg_hi = seg_base[(size_t)l + 1];
         B.fix_lo = fix_at[(size_t)l];
         B.fix_hi = fix_at[(size_t)l + 1];
+        B.hub_lo = hub_at[(size_t)l];
+        B.hub_hi = hub_at[(size_t)l + 1];
         B.done_row_lo = l == 0 ? 0 : h_rows[(size_t)l - 1].done_row_hi;
         B.done_row_hi = l == b - 1 ? n : r.done_row_hi;
     }
@@ -833,7 +887,18 @@ extern "C" int gnnpre_plan_support(const gnnpre_plan_t* P, int64_t* rowptr_out, 
 
 extern "C" void gnnpre_plan_destroy(gnnpre_plan_t* P) {
     if (!P) return;
-    cudaDeviceSynchronize();
+    // Wait for the work that still uses the plan's memory - the last device-resident call (an event on the
+    // caller's stream) and the plan's own streams - not for the whole device.
+    // (an event last recorded inside a stream capture cannot be waited for: then wait for the device)
+    if (P->last_use && cudaEventSynchronize(P->last_use) != cudaSuccess) {
+        (void)cudaGetLastError();
+        cudaDeviceSynchronize();
+    }
+    if (P->s_h2d) cudaStreamSynchronize(P->s_h2d);
+    if (P->s_compute) cudaStreamSynchronize(P->s_compute);
+    if (P->s_d2h) cudaStreamSynchronize(P->s_d2h);
+    if (P->s_struct) cudaStreamSynchronize(P->s_struct);
+    (void)cudaGetLastError();
     delete P;
 }
 

@@ -1,0 +1,232 @@
+// Register-gather segment kernel and the pieces every propagation kernel shares (the epilogue of a finished
+// row, the launch arguments, compensated addition).  Included by propagate.cu inside its unnamed namespace.
+#pragma once
+
+// The optional teleport term: a finished row r_i * sum becomes keep * (r_i * sum) + alpha * X_0[i].
+struct Teleport {
+    const float* x0;
+    int64_t ldx0;
+    float alpha, keep;  // keep = 1 - alpha
+    // fixed-weight sum of hops (zsum == nullptr: none): Z += gamma * (the value stored for this hop)
+    float* zsum;
+    int64_t ldz;
+    float gamma, gamma0;
+    int zsum_first;
+};
+
+// EP, the epilogue of a finished row: 0 = scale only; 1 = scale and teleport term; 2 = the launch also accumulates the
+// fixed-weight sum of hops (teleport decided at run time).  A compile-time switch, because the mere presence of the
+// optional code slowed the plain kernels down although its branches were never taken (the L2-resident workload by
+// 10 % for the teleport term and by 40 % for the sum).
+constexpr int kEpPlain = 0, kEpTeleport = 1, kEpSum = 2;
+template <int EP>
+__device__ __forceinline__ float4 finish_row_piece(float4 sum, float scale, const Teleport& tp, int64_t row, int q) {
+    float4 o = make_float4(sum.x * scale, sum.y * scale, sum.z * scale, sum.w * scale);
+    if (EP == kEpTeleport || (EP == kEpSum && tp.alpha != 0.f)) {
+        const float4 z = __ldg(reinterpret_cast<const float4*>(tp.x0 + row * tp.ldx0) + q);
+        o.x = fmaf(tp.keep, o.x, tp.alpha * z.x);
+        o.y = fmaf(tp.keep, o.y, tp.alpha * z.y);
+        o.z = fmaf(tp.keep, o.z, tp.alpha * z.z);
+        o.w = fmaf(tp.keep, o.w, tp.alpha * z.w);
+    }
+    if (EP == kEpSum) {  // every finished row piece passes here exactly once per hop
+        float4* zp = reinterpret_cast<float4*>(tp.zsum + row * tp.ldz) + q;
+        float4 acc;
+        if (tp.zsum_first) {
+            const float4 x = __ldg(reinterpret_cast<const float4*>(tp.x0 + row * tp.ldx0) + q);
+            acc = make_float4(tp.gamma0 * x.x, tp.gamma0 * x.y, tp.gamma0 * x.z, tp.gamma0 * x.w);
+        } else {
+            acc = *zp;
+        }
+        acc.x = fmaf(tp.gamma, o.x, acc.x);
+        acc.y = fmaf(tp.gamma, o.y, acc.y);
+        acc.z = fmaf(tp.gamma, o.z, acc.z);
+        acc.w = fmaf(tp.gamma, o.w, acc.w);
+        *zp = acc;
+    }
+    return o;
+}
+
+// Which epilogue a launch needs.
+inline int epilogue_of(const Teleport& tp) { return tp.zsum != nullptr ? kEpSum : tp.alpha != 0.f ? kEpTeleport : kEpPlain; }
+
+struct SegArgs {
+    const Segment* segs;
+    int64_t seg_lo, seg_hi;
+    const uint32_t* colx;
+    int64_t colx_base;
+    const float* x;
+    int64_t ldx;
+    float* out;
+    int64_t ldo;
+    float* scratch;
+    int64_t scratch_ld;
+    const float* rscale;
+    const float* cscale;
+    const int32_t* nzrows;
+    int32_t f4;  // float4 per row of this column tile
+    float diag_weight;  // GIN: 1 + eps
+    Teleport tp;
+};
+
+// Compensated (Kahan) addition of x into the pair (sum, comp): the low-order bits that the addition
+// drops are carried in comp.
+__device__ __forceinline__ void kahan1(float& sum, float& comp, float x) {
+    const float y = x - comp;
+    const float t = sum + y;
+    comp = (t - sum) - y;
+    sum = t;
+}
+
+__device__ __forceinline__ void kahan4(float4& sum, float4& comp, const float4& x) {
+    kahan1(sum.x, comp.x, x.x);
+    kahan1(sum.y, comp.y, x.y);
+    kahan1(sum.z, comp.z, x.z);
+    kahan1(sum.w, comp.w, x.w);
+}
+
+constexpr int kThreads = 256;
+constexpr int kMaxDevices = 64;
+
+// G lanes per segment, V float4 per lane (row width <= 4*G*V floats), U rows in flight per lane.
+//
+// Accumulation: the U rows of one step are added in a short plain fp32 chain, and that partial sum
+// enters the row's running sum by a compensated (Kahan) addition, so the rounding error of a row
+// stays at a few ulps of sum_j |w_j x_j| whatever its degree, at ~2 extra instructions per edge.
+#ifndef GNNPRE_SEG_U
+#define GNNPRE_SEG_U 8
+#endif
+#ifndef GNNPRE_SEG_MIN_BLOCKS
+#define GNNPRE_SEG_MIN_BLOCKS 3
+#endif
+template <int G, int V, int U, int OP, bool HAS_EMPTY, int EP>
+__global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
+    constexpr unsigned kFull = 0xffffffffu;
+    const int lane = threadIdx.x & 31;
+    const int gl = lane & (G - 1);
+    const int gshift = lane & ~(G - 1);
+    const unsigned glow = G == 32 ? kFull : ((1u << G) - 1u);
+    const unsigned gmask = glow << gshift;
+    const int64_t s = a.seg_lo + ((int64_t)blockIdx.x * kThreads + threadIdx.x) / G;
+
+    int64_t e = 0, e_end = 0;
+    int rank = 0, slot_head = -1, slot_tail = -1;
+    if (s < a.seg_hi) {
+        const Segment g = a.segs[s];
+        e = g.start;
+        e_end = a.segs[s + 1].start;
+        rank = g.rank;
+        slot_head = g.slot_head;
+        slot_tail = g.slot_tail;
+    }
+    // Lane gl owns float4 columns gl, gl + G, ...; lanes beyond the row's width re-read column 0 so
+    // that every load is unconditional and in bounds (their sums are never stored).
+    bool on[V];
+    const float4* xlane[V];
+    const uint32_t ldx4 = (uint32_t)(a.ldx >> 2);
+#pragma unroll
+    for (int v = 0; v < V; ++v) {
+        const int q = gl + v * G;
+        on[v] = q < a.f4;
+        xlane[v] = reinterpret_cast<const float4*>(a.x) + (on[v] ? q : 0);
+    }
+    bool head_pending = slot_head >= 0;  // the first row began in an earlier segment
+    bool open = false;                   // the last edge seen so far did not end its row
+    float4 acc[V], tot[V], cmp[V];       // this step's plain sum; the row's running sum and its compensation
+#pragma unroll
+    for (int v = 0; v < V; ++v) acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+    while (__any_sync(kFull, e < e_end)) {
+        // ---- this chunk's edges: lane gl of the group owns edge e + gl; lanes past the end hold 0,
+        // a valid column without a row-end mark
+        const int64_t left = e_end - e;
+        const int cnt = left >= G ? G : (left > 0 ? (int)left : 0);
+        uint32_t c = 0;
+        if (gl < cnt) c = a.colx[e + gl - a.colx_base];
+        const unsigned ends = (__ballot_sync(kFull, (c & kRowEndBit) != 0) >> gshift) & glow;
+        int my_row = rank + __popc(ends & ((1u << gl) - 1u));
+        float my_r = 1.f, w = 1.f;
+        if (c & kRowEndBit) {
+            if (HAS_EMPTY) my_row = a.nzrows[my_row];
+            if (OP != GNNPRE_OP_GIN_SUM) my_r = a.rscale[my_row];
+        }
+        if (OP == GNNPRE_OP_GCN_SYM) {
+            w = a.cscale[c & ~kRowEndBit];
+        } else if (OP == GNNPRE_OP_GIN_SUM) {
+            w = (int)(c & ~kRowEndBit) == my_row ? a.diag_weight : 1.f;  // every row owns its self-loop: rank == row
+        }
+        if (cnt > 0) open = (__shfl_sync(gmask, c, gshift + cnt - 1) & kRowEndBit) == 0;
+        const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
+
+        // ---- gather and accumulate, U rows in flight
+        for (int t0 = 0; t0 < cnt_max; t0 += U) {
+            float4 x[U][V];
+            uint32_t craw[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                craw[u] = __shfl_sync(kFull, c, t0 + u, G);
+                const uint64_t off = (uint64_t)(craw[u] & ~kRowEndBit) * ldx4;
+#pragma unroll
+                for (int v = 0; v < V; ++v) x[u][v] = __ldg(xlane[v] + off);
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int t = t0 + u;
+                if (t < cnt) {
+                    if (OP == GNNPRE_OP_SAGE_MEAN) {
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            acc[v].x += x[u][v].x; acc[v].y += x[u][v].y;
+                            acc[v].z += x[u][v].z; acc[v].w += x[u][v].w;
+                        }
+                    } else {
+                        const float ww = __shfl_sync(gmask, w, gshift + t);
+#pragma unroll
+                        for (int v = 0; v < V; ++v) {
+                            acc[v].x = fmaf(ww, x[u][v].x, acc[v].x); acc[v].y = fmaf(ww, x[u][v].y, acc[v].y);
+                            acc[v].z = fmaf(ww, x[u][v].z, acc[v].z); acc[v].w = fmaf(ww, x[u][v].w, acc[v].w);
+                        }
+                    }
+                }
+                if (craw[u] & kRowEndBit) {
+                    // last edge of a row (never set on a padding lane): the whole group arrives here together
+                    const int row = __shfl_sync(gmask, my_row, gshift + t);
+                    const float r = __shfl_sync(gmask, my_r, gshift + t);
+                    const bool partial = head_pending;  // the row began earlier: leave the sum for the fix-up
+                    head_pending = false;
+                    float* dst = partial ? a.scratch + (int64_t)slot_head * a.scratch_ld : a.out + (int64_t)row * a.ldo;
+#pragma unroll
+                    for (int v = 0; v < V; ++v) {
+                        kahan4(tot[v], cmp[v], acc[v]);
+                        if (on[v])
+                            reinterpret_cast<float4*>(dst)[gl + v * G] =
+                                partial ? tot[v] : finish_row_piece<EP>(tot[v], r, a.tp, row, gl + v * G);
+                        acc[v] = tot[v] = cmp[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            }
+            if (t0 < cnt) {  // this step's plain sum joins the row's compensated sum (never on a padding
+                             // step: the result must not depend on which segment shares the warp)
+#pragma unroll
+                for (int v = 0; v < V; ++v) {
+                    kahan4(tot[v], cmp[v], acc[v]);
+                    acc[v] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+            }
+        }
+        rank += __popc(ends);
+        e += G;
+    }
+
+    // ---- the row holding the last edge continues in the next segment
+    if (open) {
+        const int slot = head_pending ? slot_head : slot_tail;
+        if (slot >= 0) {
+            float* dst = a.scratch + (int64_t)slot * a.scratch_ld;
+#pragma unroll
+            for (int v = 0; v < V; ++v)
+                if (on[v]) reinterpret_cast<float4*>(dst)[gl + v * G] = tot[v];
+        }
+    }
+}
+

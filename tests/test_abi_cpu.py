@@ -42,7 +42,7 @@ def test_struct_layouts_match_header(binding):
     assert ctypes.sizeof(binding.gnnpre_plan_opts_t) == 48
     assert ctypes.sizeof(binding.gnnpre_block_info_t) == 32
     assert ctypes.sizeof(binding.gnnpre_plan_info_t) == 152
-    assert ctypes.sizeof(binding.gnnpre_stats_t) == 64 * 4 + 8 + 32
+    assert ctypes.sizeof(binding.gnnpre_stats_t) == 64 * 4 + 8 + 32 + 16
 
 
 def test_status_strings(binding):

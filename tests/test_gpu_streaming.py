@@ -1,0 +1,222 @@
+"""GPU tests of the host-operand pipeline's second schedule (whole hop matrices on the device, narrow-first
+column panels), of the status query for asynchronous calls, of host-side allocation-failure injection and of
+the operand-overlap checks.  Nothing here faults, traps or hangs a device."""
+import numpy as np
+import pytest
+import torch
+
+import gnnpre_inputs as gi
+from parity_util import check_all_hops, to_np
+
+pytestmark = pytest.mark.gpu
+
+OPS = (0, 1, 2)
+EPS = 0.1
+
+
+@pytest.fixture(scope="module")
+def B():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2207_12000_b200 import binding
+    return binding
+
+
+def dev(g):
+    return g.rowptr.cuda(), g.colidx.cuda()
+
+
+def pinned(n, ld, fill=None):
+    t = torch.empty((n, ld), dtype=torch.float32).pin_memory()
+    if fill is not None:
+        t.fill_(fill)
+    return t
+
+
+@pytest.mark.parametrize("op", OPS)
+@pytest.mark.parametrize("F,K,csr_on_host", [(128, 2, False), (128, 2, True), (256, 3, False), (160, 1, False)])
+def test_panel_schedule_equals_resident_and_oracle(B, op, F, K, csr_on_host):
+    """Host X and host out[] with room for K + 1 whole matrices: the call runs the panel schedule (3, 4 and 4
+    upload slabs for F = 128, 256, 160), edge blocks streamed or resident.  Every column is an independent
+    product and the segment kernels add a row's edges in the same order whatever the tile width, so for
+    F <= 128 the result equals the device-resident run of the same (b, segment size) bit for bit; wider rows
+    agree to rounding (the resident run sums 256-column tiles in steps of four edges).  All hops are checked
+    against the fp64 oracle, pad columns of the host matrices stay untouched, and a second call reuses the
+    buffers."""
+    g = gi.rmat(30000, 250000, 41, directed_candidates=True)
+    rp_np, ci_np = g.rowptr.numpy(), g.colidx.numpy()
+    drp, dci = dev(g)
+    X = gi.normal_matrix(g.n, F, 9, device="cuda")
+    rp, ci = (g.rowptr.pin_memory(), g.colidx.pin_memory()) if csr_on_host else (drp, dci)
+    plan = B.gnnpre_build_plan(rp, ci, op, F, gin_eps=EPS, force_blocks=3, segment_edges=64,
+                               operands_mem=B.GNNPRE_MEM_HOST)
+    info = plan.info()
+    assert info["c"] == 2 and info["structure_mem"] == (1 if csr_on_host else 0)
+    ld = F + 32  # rows of the host matrices start on 128-byte boundaries
+    Xh = pinned(g.n, ld, 7.0)
+    Xh[:, :F].copy_(X)
+    obuf = [pinned(g.n, ld, -3.0) for _ in range(K)]
+    ref_plan = B.gnnpre_build_plan(drp, dci, op, F, gin_eps=EPS, force_blocks=3, segment_edges=64)
+    ref, _ = B.gnnpre_propagate(ref_plan, X, K)
+    torch.cuda.synchronize()
+    for rep in range(2):
+        outs, st = B.gnnpre_propagate(plan, Xh[:, :F], K, [o[:, :F] for o in obuf], want_stats=True)
+        assert st.schedule == B.GNNPRE_SCHEDULE_PANELS
+        assert st.upload_slabs == {128: 3, 256: 4, 160: 4}[F]
+        assert st.d2h_bytes == 4 * g.n * F * K and st.h2d_bytes >= 4 * g.n * F
+        assert st.startup_ms > 0 and st.drain_ms > 0
+        for k in range(K):
+            assert bool((obuf[k][:, F:] == -3.0).all())
+            if F <= 128:
+                assert torch.equal(outs[k], ref[k].cpu()), (k, rep)
+        check_all_hops(op, EPS, rp_np, ci_np, to_np(X), outs)
+        for o in obuf:
+            o[:, :F].fill_(-1.0)
+    assert plan.info()["device_bytes"] >= (K + 1) * g.n * F * 4
+    plan.close()
+    ref_plan.close()
+
+
+def test_panel_schedule_is_left_when_its_conditions_fail(B):
+    """Forced c, rows off the 128-byte grid, a width that is not a multiple of 32, or a budget without room for
+    the whole matrices: the call falls back to Algorithm 1's equal slabs and still matches the oracle."""
+    g = gi.rmat(20000, 160000, 43, directed_candidates=True)
+    rp_np, ci_np = g.rowptr.numpy(), g.colidx.numpy()
+    K = 2
+    cases = [dict(F=128, ld=128, kw=dict(force_col_slabs=2)),
+             dict(F=128, ld=132, kw=dict()),
+             dict(F=136, ld=160, kw=dict()),
+             dict(F=128, ld=128, kw=dict(budget_bytes=2 * g.n * 128 * 4 + 16 * g.n + 4 * (g.nnz + g.n) + 8 * (g.n + 1) + 4096))]
+    for case in cases:
+        F, ld = case["F"], case["ld"]
+        X = gi.normal_matrix(g.n, F, 10, device="cuda")
+        plan = B.gnnpre_build_plan(*dev(g), 0, F, operands_mem=B.GNNPRE_MEM_HOST, **case["kw"])
+        Xh = pinned(g.n, ld, 0.0)
+        Xh[:, :F].copy_(X)
+        outs, st = B.gnnpre_propagate(plan, Xh[:, :F], K, [pinned(g.n, ld)[:, :F] for _ in range(K)], want_stats=True)
+        assert st.schedule == B.GNNPRE_SCHEDULE_SLABS, case
+        check_all_hops(0, 0.0, rp_np, ci_np, to_np(X), outs)
+        plan.close()
+
+
+def test_panel_schedule_with_teleport_term(B):
+    """The personalised-PageRank recurrence reads X_0's columns in every hop: they stay on the device whole."""
+    import oracle as orc
+    from parity_util import TOL, hop_error
+    g = gi.rmat(15000, 120000, 44, directed_candidates=True)
+    F, K, alpha = 128, 3, 0.15
+    X = gi.normal_matrix(g.n, F, 11)
+    plan = B.gnnpre_build_plan(*dev(g), 0, F, operands_mem=B.GNNPRE_MEM_HOST, teleport_alpha=alpha)
+    outs, st = B.gnnpre_propagate(plan, X.pin_memory(), K, [pinned(g.n, F) for _ in range(K)], want_stats=True)
+    assert st.schedule == B.GNNPRE_SCHEDULE_PANELS
+    want = orc.propagate_teleport(0, 0.0, alpha, g.rowptr.numpy(), g.colidx.numpy(), X.numpy(), K)
+    for k in range(K):
+        assert hop_error(outs[k].numpy(), want[k]) <= TOL
+    plan.close()
+
+
+def test_status_query_reports_a_timed_out_wait_of_an_asynchronous_call_once(B):
+    """A device-resident call without stats only enqueues work, so a wait that ran out inside one of its kernels
+    is learnt through gnnpre_plan_status.  The self-test kernel stands in for such a kernel: it polls a barrier
+    nothing completes, gives up after its limit and raises the plan's error word (no fault, the device stays
+    usable).  The query reports the timeout exactly once, and the plan then propagates correctly."""
+    g = gi.erdos_renyi(3000, 20000, 23)
+    plan = B.gnnpre_build_plan(*dev(g), 0, 128)
+    assert B.gnnpre_plan_status(plan) == 0
+    B.gnnpre_selftest_wait_timeout_async(plan, 100)
+    X = gi.normal_matrix(g.n, 128, 2, device="cuda")
+    outs, _ = B.gnnpre_propagate(plan, X, 2)  # asynchronous, returns GNNPRE_OK whatever happens on the device
+    assert B.gnnpre_plan_status(plan) == -8
+    assert B.gnnpre_plan_status(plan) == 0
+    outs, _ = B.gnnpre_propagate(plan, X, 2)
+    assert B.gnnpre_plan_status(plan) == 0
+    check_all_hops(0, 0.0, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), outs)
+    plan.close()
+
+
+def test_injected_allocation_failures_leave_nothing_behind(B):
+    """Host-side failure injection: the N-th allocation of a plan build (device), of a host-structure build
+    (page-locked memory) and of a streamed call is reported as failed.  Every failed build returns no plan and
+    the device's free memory goes back to where it was; a failed streamed call leaves the plan usable.  The
+    hook disarms itself after one failure and the next build succeeds."""
+    g = gi.rmat(20000, 160000, 45, directed_candidates=True)
+    drp, dci = dev(g)
+    F = 128
+    torch.cuda.synchronize()
+    B.gnnpre_build_plan(drp, dci, 1, F, force_blocks=3).close()  # warm-up: lazily loaded kernels take memory once
+    free0 = torch.cuda.mem_get_info()[0]
+    fails = 0
+    for N in range(64):
+        B.gnnpre_inject_alloc_failure(N, -1)
+        try:
+            plan = B.gnnpre_build_plan(drp, dci, 1, F, force_blocks=3)
+        except B.GnnpreError as e:
+            assert e.status == -4  # GNNPRE_ERR_OOM_DEVICE
+            fails += 1
+            assert torch.cuda.mem_get_info()[0] == free0
+            continue
+        plan.close()
+        break
+    else:
+        pytest.fail("a plan build made more than 64 device allocations")
+    B.gnnpre_inject_alloc_failure(-1, -1)
+    assert fails >= 10  # per-node arrays, E, row pointers, segment tables, scan temporaries, scratch ...
+    assert torch.cuda.mem_get_info()[0] == free0
+
+    # page-locked host memory: the plan's copy of E when the structure stays on the host
+    rp_h, ci_h = g.rowptr.pin_memory(), g.colidx.pin_memory()
+    B.gnnpre_inject_alloc_failure(-1, 0)
+    with pytest.raises(B.GnnpreError) as ei:
+        B.gnnpre_build_plan(rp_h, ci_h, 0, F, force_blocks=4, operands_mem=B.GNNPRE_MEM_HOST)
+    assert ei.value.status == -5  # GNNPRE_ERR_OOM_HOST
+    assert torch.cuda.mem_get_info()[0] == free0
+
+    # a streamed call: slab buffers are allocated on first use
+    plan = B.gnnpre_build_plan(rp_h, ci_h, 0, F, force_blocks=4, force_col_slabs=2, operands_mem=B.GNNPRE_MEM_HOST)
+    X = gi.normal_matrix(g.n, F, 12)
+    Xh, outs = X.pin_memory(), [pinned(g.n, F) for _ in range(2)]
+    fails = 0
+    for N in range(8):  # buffers that one attempt managed to allocate are kept, so each attempt gets further
+        B.gnnpre_inject_alloc_failure(N, -1)
+        try:
+            B.gnnpre_propagate(plan, Xh, 2, outs)
+        except B.GnnpreError as e:
+            assert e.status == -4
+            fails += 1
+            continue
+        break
+    B.gnnpre_inject_alloc_failure(-1, -1)
+    assert fails >= 2
+    B.gnnpre_propagate(plan, Xh, 2, outs)  # the same plan, now with all four slab buffers
+    check_all_hops(0, 0.0, g.rowptr.numpy(), g.colidx.numpy(), X.numpy(), outs)
+    plan.close()
+    assert torch.cuda.mem_get_info()[0] == free0
+
+
+def test_overlapping_operands_are_rejected_and_column_views_accepted(B):
+    """X, out[] and Z are checked for shared elements, not only for equal base pointers; the hops of one call
+    may be column views of one wide buffer (concatenated hops, as JKNet's COMB wants them)."""
+    g = gi.erdos_renyi(2000, 12000, 46)
+    F, K = 64, 3
+    plan = B.gnnpre_build_plan(*dev(g), 0, F)
+    X = gi.normal_matrix(g.n, F, 13, device="cuda")
+    big = torch.empty((g.n + 8, F), device="cuda")
+    with pytest.raises(B.GnnpreError) as ei:  # two hops that share all but four rows
+        B.gnnpre_propagate(plan, X, 2, [big[:g.n], big[4:g.n + 4]])
+    assert ei.value.status == -1
+    xbig = torch.zeros((g.n + 1, F), device="cuda")
+    with pytest.raises(B.GnnpreError):  # out[0] starts one row into X
+        B.gnnpre_propagate(plan, xbig[:g.n], 1, [xbig[1:]])
+    wide = torch.empty((g.n, 2 * F), device="cuda")
+    with pytest.raises(B.GnnpreError):  # column views that share 16 columns
+        B.gnnpre_propagate(plan, X, 2, [wide[:, :F], wide[:, F - 16:2 * F - 16]])
+    cat = torch.full((g.n, K * F), float("nan"), device="cuda")
+    outs, _ = B.gnnpre_propagate(plan, X, K, [cat[:, k * F:(k + 1) * F] for k in range(K)])
+    torch.cuda.synchronize()
+    check_all_hops(0, 0.0, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), [o.contiguous() for o in outs])
+    Z = torch.empty((g.n, F), device="cuda")
+    with pytest.raises(B.GnnpreError):  # Z inside a hop buffer
+        B.gnnpre_propagate_weighted(plan, X, [1.0, 0.5, 0.25], out=[cat[:, :F], cat[:, F:2 * F]], Z=cat[:, 16:F + 16])
+    B.gnnpre_propagate_weighted(plan, X, [1.0, 0.5, 0.25], out=[cat[:, :F], cat[:, F:2 * F]], Z=Z)
+    assert B.gnnpre_plan_status(plan) == 0
+    plan.close()

@@ -49,6 +49,38 @@ def test_static_hop_matches_planned_hop_twice_in_a_row(B, op):
         plan.close()
 
 
+def test_static_hop_wide_rows_longer_segments_and_no_allocation(B):
+    """Rows of 256 and 512 columns (two and four 128-bit pieces per lane) on a graph large enough that the
+    segments must grow beyond 64 edges for their partial sums to fit the fixed array (3.2 M edges at F = 256:
+    segments of 128 edges).  After the first call the device's free memory is read before and after each call:
+    the entry point must not change it."""
+    import ctypes
+    g = gi.rmat(100000, 1600000, 22, directed_candidates=False)
+    assert 2 * ((g.nnz + 63) // 64) * 256 * 4 > 64 << 20  # 64-edge segments would not fit
+    drp, dci = g.rowptr.cuda(), g.colidx.cuda()
+    rp, ci = g.rowptr.numpy(), g.colidx.numpy()
+    for F, op in ((256, 0), (512, 1), (132, 2)):
+        X = gi.normal_matrix(g.n, F, 5, device="cuda")
+        out = torch.empty_like(X)
+        want = orc.propagate(op, 0.1, rp, ci, to_np(X), 1)[0]
+        B.gnnpre_hop_static(drp, dci, op, X, out, gin_eps=0.1)  # may be the first call on this device: set-up
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        for _ in range(2):
+            out.fill_(7.0)
+            B.gnnpre_hop_static(drp, dci, op, X, out, gin_eps=0.1)
+            torch.cuda.synchronize()
+            assert torch.cuda.mem_get_info()[0] == free_before
+            assert hop_error(to_np(out), want) <= TOL
+    # a problem whose partial sums cannot fit whatever the segment length: refused before anything is launched
+    # (the edge count is only read, never followed, so a made-up one is safe to pass)
+    csr = B.gnnpre_csr_t(g.n, 1 << 35, drp.data_ptr(), dci.data_ptr(), B.GNNPRE_MEM_DEVICE)
+    X = torch.zeros((g.n, 512), device="cuda")
+    rc = B._lib.gnnpre_hop_static(ctypes.byref(csr), 0, 0.0, 512, X.data_ptr(), 512, torch.empty_like(X).data_ptr(), 512,
+                                  torch.cuda.current_stream().cuda_stream)
+    assert rc == -11
+
+
 def test_static_hop_edge_cases_and_limits(B):
     g = gi.from_edge_list(6, [])  # no edges: only self-loop terms
     X = gi.normal_matrix(6, 8, 3, device="cuda")
