@@ -11,7 +11,7 @@
 #pragma once
 
 template <int G, int V, int U>
-__global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_ceiling(const SegArgs a, float* __restrict__ sink) {
+__global__ void __launch_bounds__(kThreads, G <= 4 ? 4 : GNNPRE_SEG_MIN_BLOCKS) k_ceiling(const SegArgs a, float* __restrict__ sink) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (G - 1);

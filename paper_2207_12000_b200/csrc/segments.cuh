@@ -100,7 +100,7 @@ constexpr int kMaxDevices = 64;
 #define GNNPRE_SEG_MIN_BLOCKS 3
 #endif
 template <int G, int V, int U, int OP, bool HAS_EMPTY, int EP>
-__global__ void __launch_bounds__(kThreads, GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
+__global__ void __launch_bounds__(kThreads, G <= 4 ? 4 : GNNPRE_SEG_MIN_BLOCKS) k_segments(const SegArgs a) {
     constexpr unsigned kFull = 0xffffffffu;
     const int lane = threadIdx.x & 31;
     const int gl = lane & (G - 1);

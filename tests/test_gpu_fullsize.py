@@ -81,9 +81,10 @@ def test_config5_scaled_streamed_with_budget(B):
     assert st.d2h_bytes == 4 * g.n * F * K
     assert st.h2d_bytes >= 4 * g.n * F + 4 * m  # X once, and E at least once
     # Eq. 12 is a model: what the plan really holds on the device after a streamed call (edge-block staging
-    # buffers, four slab buffers, per-node arrays, row pointers, segment tables) stays within 10 % of the budget
+    # buffers, four slab buffers, per-node arrays, row pointers, segment tables, scratch rows) exceeds the budget by
+    # 8.3 % at this size (measured; 1.9 % at 1/16 scale, 0.2 % at 1/4 scale: the tables grow slower than the matrices)
     used = plan.info()["device_bytes"]
-    assert used <= 1.10 * budget, (used, budget)
+    assert used <= 1.09 * budget, (used, budget)
     ref_plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, force_blocks=info["b"], force_col_slabs=info["c"],
                                    segment_edges=info["segment_edges"])
     ref, _ = B.gnnpre_propagate(ref_plan, X, K)
@@ -210,7 +211,7 @@ def test_config5_quarter_scale_streamed_sampled(B):
     _, st = B.gnnpre_propagate(plan_b, Xh, K, outs_b, want_stats=True)
     assert st.schedule == B.GNNPRE_SCHEDULE_SLABS
     assert st.h2d_bytes == 4 * n * F + 4 * m * K * info_b["c"]  # X once; E once per slab and hop
-    assert plan_b.info()["device_bytes"] <= 1.10 * budget
+    assert plan_b.info()["device_bytes"] <= 1.01 * budget  # the budget model against what is really held: +0.2 % here
     ref_plan = B.gnnpre_build_plan(g.rowptr, g.colidx, w.op, F, force_blocks=4, force_col_slabs=4,
                                    segment_edges=info_b["segment_edges"], flags=B.GNNPRE_FLAG_LAUNCH_PER_BLOCK)
     ref, _ = B.gnnpre_propagate(ref_plan, X, K)
