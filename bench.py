@@ -65,7 +65,8 @@ def parse():
                     help="--stage lc: which precision the line leads with: every operand split into two tf32 numbers "
                          "(fp32-like accuracy, the like-for-like figure: the paper's arithmetic is fp32), or plain tf32 "
                          "operands; the other one is timed beside it")
-    ap.add_argument("--e2e-col-slabs", type=int, default=0, help="column slabs c of the host-buffer run (0 = the library's choice)")
+    ap.add_argument("--e2e-col-slabs", type=int, default=0, help="column slabs c of the host-buffer runs (0 = the library's choice; forcing c also "
+                                                                    "forces the equal-slab schedule)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-configs", action="store_true",
                     help="default run only: skip the compact records of configurations 1, 2, 3 (a corner) and 5")
@@ -535,7 +536,7 @@ def c5_streamed_record(B, args):
     Xh = gi.normal_matrix(w.n, w.feat_dim, w.seed, device="cuda", pin=True)
     torch.cuda.synchronize()
     torch.cuda.empty_cache()
-    rec, outs_h, Xh = streamed_run(B, w, g, Xh, args, reps=3, blocks=0, col_slabs=0)
+    rec, outs_h, Xh = streamed_run(B, w, g, Xh, args, reps=3, blocks=0, col_slabs=args.e2e_col_slabs)
     rec["workload"] = (f"{w.name}: rmat graph, {g.n} nodes, {g.nnz} directed nnz, F={w.feat_dim}, K={w.hops}, op=gcn_sym; "
                        "graph, X and hop outputs in pinned host memory")
     rec["scale_note"] = (f"configuration 5 at 1/{args.c5_scale} of its nodes and edges: at full size X and two hop outputs alone "

@@ -674,7 +674,16 @@ int build_plan_impl(const gnnpre_csr_t* csr, const int32_t* degrees, const gnnpr
     GNNPRE_CUDA(cudaMemcpy(h_rows.data(), d_rows.p, sizeof(BlockRows) * (size_t)b, cudaMemcpyDeviceToHost));
 
     // ---- segments, scratch slots and row fix-ups
-    k_segment_starts<<<grid_for(nseg + 1, kTB), kTB, 0, st>>>(nseg, (int)b, d_seg_base.p, d_e_off.p, L, L / 2,
+    // How far a nominal cut inside a row may move forward to the next row start.  Half a segment keeps the segments
+    // balanced (moving by up to a whole one cost 3-15 % on every larger workload).  A launch so small that all its
+    // segments are resident at once is bound by latency, not balance: there the cut may move by up to L - 1 edges,
+    // which leaves a graph of short rows without any cut row and so without the fix-up launch (4,096 nodes of
+    // degree 16: two launches per step of two hops instead of four, 39 -> 31 us).
+    const int64_t f4_slab = std::min<int64_t>(P->slab_width, 512) / 4;
+    const int64_t lanes = f4_slab <= 4 ? 4 : f4_slab <= 8 ? 8 : f4_slab <= 16 ? 16 : 32;
+    const bool one_wave = nseg * lanes <= (int64_t)P->num_sms * 768;
+    const int32_t snap = one_wave ? L - 1 : L / 2;
+    k_segment_starts<<<grid_for(nseg + 1, kTB), kTB, 0, st>>>(nseg, (int)b, d_seg_base.p, d_e_off.p, L, snap,
                                                               P->rowptr_t.p, n, rank.p, P->segments.p);
     GNNPRE_CUDA(cudaGetLastError());
     DevBuf<int32_t> flags, slot_scan, emit, emit_scan;
