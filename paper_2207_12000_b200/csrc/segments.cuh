@@ -155,16 +155,30 @@ __global__ void __launch_bounds__(kThreads, G <= 4 ? 4 : GNNPRE_SEG_MIN_BLOCKS) 
         } else if (OP == GNNPRE_OP_GIN_SUM) {
             w = (int)(c & ~kRowEndBit) == my_row ? a.diag_weight : 1.f;  // every row owns its self-loop: rank == row
         }
-        if (cnt > 0) open = (__shfl_sync(gmask, c, gshift + cnt - 1) & kRowEndBit) == 0;
+        if (cnt > 0) open = ((ends >> (cnt - 1)) & 1u) == 0;  // the chunk's last edge does not end its row
         const int cnt_max = G == 32 ? cnt : __reduce_max_sync(kFull, cnt);
 
         // ---- gather and accumulate, U rows in flight
         for (int t0 = 0; t0 < cnt_max; t0 += U) {
             float4 x[U][V];
             uint32_t craw[U];
+            // Four-lane groups also hand every edge's row and row scale around ahead of time: with eight groups in a
+            // warp a row ends somewhere in almost every step, and the two shuffles under a partial mask that a row end
+            // otherwise costs are dearer than two plain ones per edge (measured: faster at G = 4, slower at G = 8, 16).
+            constexpr bool kRowsAhead = G == 4;
+            int rowv[U];
+            float rv[U];
+            float wv[U];  // the edges' weights, handed to the group together with their column entries (whole-warp
+                          // shuffles outside any branch: a shuffle under a partial mask inside the per-edge
+                          // condition below cost the weighted operators half again the time of the unweighted one)
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 craw[u] = __shfl_sync(kFull, c, t0 + u, G);
+                if (OP != GNNPRE_OP_SAGE_MEAN) wv[u] = __shfl_sync(kFull, w, t0 + u, G);
+                if (kRowsAhead) {
+                    rowv[u] = __shfl_sync(kFull, my_row, t0 + u, G);
+                    rv[u] = __shfl_sync(kFull, my_r, t0 + u, G);
+                }
                 const uint64_t off = (uint64_t)(craw[u] & ~kRowEndBit) * ldx4;
 #pragma unroll
                 for (int v = 0; v < V; ++v) x[u][v] = __ldg(xlane[v] + off);
@@ -180,7 +194,7 @@ __global__ void __launch_bounds__(kThreads, G <= 4 ? 4 : GNNPRE_SEG_MIN_BLOCKS) 
                             acc[v].z += x[u][v].z; acc[v].w += x[u][v].w;
                         }
                     } else {
-                        const float ww = __shfl_sync(gmask, w, gshift + t);
+                        const float ww = wv[u];
 #pragma unroll
                         for (int v = 0; v < V; ++v) {
                             acc[v].x = fmaf(ww, x[u][v].x, acc[v].x); acc[v].y = fmaf(ww, x[u][v].y, acc[v].y);
@@ -190,8 +204,8 @@ __global__ void __launch_bounds__(kThreads, G <= 4 ? 4 : GNNPRE_SEG_MIN_BLOCKS) 
                 }
                 if (craw[u] & kRowEndBit) {
                     // last edge of a row (never set on a padding lane): the whole group arrives here together
-                    const int row = __shfl_sync(gmask, my_row, gshift + t);
-                    const float r = __shfl_sync(gmask, my_r, gshift + t);
+                    const int row = kRowsAhead ? rowv[u] : __shfl_sync(gmask, my_row, gshift + t);
+                    const float r = kRowsAhead ? rv[u] : __shfl_sync(gmask, my_r, gshift + t);
                     const bool partial = head_pending;  // the row began earlier: leave the sum for the fix-up
                     head_pending = false;
                     float* dst = partial ? a.scratch + (int64_t)slot_head * a.scratch_ld : a.out + (int64_t)row * a.ldo;
