@@ -143,10 +143,11 @@ def profiled_traffic(workload_name):
 
 
 def kernel_source_hash():
-    """sha256 over the files that hold the segment kernels (what an ncu capture of them depends on)."""
+    """sha256 over the files that hold the bulk-copy segment kernel and the pieces it shares with the others (what an
+    ncu capture of it depends on)."""
     import hashlib
     cur = hashlib.sha256()
-    for f in ("segments.cuh", "segments_tma.cuh"):
+    for f in ("segments_common.cuh", "segments_tma.cuh"):
         cur.update(open(os.path.join(ROOT, "paper_2207_12000_b200", "csrc", f), "rb").read())
     return cur.hexdigest()
 

@@ -16,7 +16,7 @@ NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", 
 def _inputs():
     src = [os.path.join(HERE, "csrc", s) for s in SOURCES]
     hdr = [os.path.join(HERE, "csrc", "gnnpre_internal.cuh"), os.path.join(HERE, "csrc", "segments_tma.cuh"),
-           os.path.join(HERE, "csrc", "segments.cuh"), os.path.join(HERE, "csrc", "fixups.cuh"), os.path.join(HERE, "csrc", "ceiling.cuh"),
+           os.path.join(HERE, "csrc", "segments.cuh"), os.path.join(HERE, "csrc", "segments_common.cuh"), os.path.join(HERE, "csrc", "fixups.cuh"), os.path.join(HERE, "csrc", "ceiling.cuh"),
            os.path.join(ROOT, "include", "gnnpre.h")]
     return src, hdr
 

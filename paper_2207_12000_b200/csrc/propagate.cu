@@ -19,6 +19,7 @@ namespace gnnpre {
 
 namespace {
 
+#include "segments_common.cuh"
 #include "segments.cuh"
 #include "segments_tma.cuh"
 
