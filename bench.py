@@ -205,7 +205,7 @@ def oracle_sample(w, g_cpu, X_cpu, target_seconds, got=None):
     diag = 0 if w.op == gi.OP_SAGE else 1
     probe_rows = max(1, n // 256)
     t0 = time.perf_counter()
-    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(probe_rows))
+    orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(probe_rows), want_abs=bool(got))
     t_probe = time.perf_counter() - t0
     probe_edges = int(rp[probe_rows]) + diag * probe_rows
     rate = probe_edges / max(t_probe, 1e-6)
@@ -214,7 +214,7 @@ def oracle_sample(w, g_cpu, X_cpu, target_seconds, got=None):
     rows = n if want_edges >= total_edges else int(np.searchsorted(rp, want_edges))
     rows = max(1, min(n, rows))
     t0 = time.perf_counter()
-    y, scale = orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(rows))
+    y, scale = orc.hop_rows_f32(w.op, w.gin_eps, rp, ci, X_cpu, np.arange(rows), want_abs=bool(got))  # |A^||X| only for the check
     t = time.perf_counter() - t0
     edges = int(rp[rows]) + diag * rows
     out = {"value": edges * X_cpu.shape[1] / t, "unit": UNIT, "cores": orc.num_threads(), "kind": "oracle",
