@@ -395,6 +395,19 @@ int gnnpre_lc_selftest_wait_timeout(const float* hop, int64_t n, int64_t feat_di
  */
 int gnnpre_gather_ceiling(gnnpre_plan_t* plan, const float* X, int64_t ldx, float* sink, void* stream);
 
+/*
+ * The narrow-first panel schedule of gnnpre_propagate for host X and host out[] (see there), as data: which column
+ * slabs X travels in and, in launch order, which hop runs on which columns and which columns of that hop's matrix
+ * leave for the host once its edge blocks finish.  Host only, no device needed; exposed so that the schedule's
+ * invariants can be checked without a GPU.
+ *   feat_dim    F, a multiple of 32;  slab_width  the plan's slab width (>= 64; no slab or job is wider);  K hops
+ *   jobs_out    6 int32 per job: hop k (1-based), first column, one past the last column, index of the upload slab
+ *               the job waits for (-1: none), first and one-past-last column drained after it (equal: nothing)
+ *   max_jobs    capacity of jobs_out in jobs; num_jobs_out receives the real count, num_slabs_out the slab count
+ */
+int gnnpre_describe_panels(int64_t feat_dim, int64_t slab_width, int32_t K, int32_t* jobs_out, int32_t max_jobs,
+                           int32_t* num_slabs_out, int32_t* num_jobs_out);
+
 /* Eq. 12 on its own (exposed for parity with the exhaustive search):
  * least b*c with ceil(beta_S B_S / b) + ceil(beta_X B_X / c) + B_fixed <= B_GPU, 1 <= b <= max_b, 1 <= c <= max_c;
  * ties towards smaller c, then smaller b.  BUDGET_TOO_SMALL if infeasible.  Host only. */

@@ -98,6 +98,7 @@ def _load() -> ctypes.CDLL:
     lib.gnnpre_selftest_wait_timeout_async.argtypes = [p, ctypes.c_uint32, p]
     lib.gnnpre_plan_status.argtypes = [p, p]
     lib.gnnpre_gather_ceiling.argtypes = [p, p, i64, p, p]
+    lib.gnnpre_describe_panels.argtypes = [i64, i64, i32, p, i32, ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.gnnpre_inject_alloc_failure.argtypes = [i64, i64]
     lib.gnnpre_plan_destroy.argtypes = [p]
     lib.gnnpre_plan_destroy.restype = None
@@ -375,6 +376,19 @@ def gnnpre_gather_ceiling(plan: Plan, X: torch.Tensor, sink: torch.Tensor | None
     return sink
 
 
+def gnnpre_describe_panels(feat_dim: int, slab_width: int, K: int):
+    """(number of upload slabs, list of jobs) of the narrow-first panel schedule; a job is a dict with keys
+    k, lo, hi, upload, drain_lo, drain_hi.  Host only."""
+    ns, nj = ctypes.c_int32(), ctypes.c_int32()
+    _check(_lib.gnnpre_describe_panels(feat_dim, slab_width, K, None, 0, ctypes.byref(ns), ctypes.byref(nj)),
+           "gnnpre_describe_panels")
+    buf = (ctypes.c_int32 * (6 * max(nj.value, 1)))()
+    _check(_lib.gnnpre_describe_panels(feat_dim, slab_width, K, buf, nj.value, ctypes.byref(ns), ctypes.byref(nj)),
+           "gnnpre_describe_panels")
+    keys = ("k", "lo", "hi", "upload", "drain_lo", "drain_hi")
+    return ns.value, [dict(zip(keys, buf[6 * i:6 * i + 6])) for i in range(nj.value)]
+
+
 def gnnpre_inject_alloc_failure(device_countdown: int = -1, host_countdown: int = -1) -> None:
     """Test hook: the library's (countdown + 1)-th next allocation of that kind is reported as failed; -1 disarms."""
     _check(_lib.gnnpre_inject_alloc_failure(device_countdown, host_countdown), "gnnpre_inject_alloc_failure")
@@ -398,5 +412,5 @@ def exported_symbols():
     return ["gnnpre_degrees", "gnnpre_build_plan", "gnnpre_plan_info", "gnnpre_plan_block", "gnnpre_plan_scales",
             "gnnpre_plan_support", "gnnpre_propagate", "gnnpre_propagate_weighted", "gnnpre_hop_static", "gnnpre_lc_first_layer", "gnnpre_lc_selftest_wait_timeout", "gnnpre_normalize",
             "gnnpre_solve_normalisation_blocks", "gnnpre_selftest_wait_timeout", "gnnpre_selftest_wait_timeout_async",
-            "gnnpre_plan_status", "gnnpre_inject_alloc_failure", "gnnpre_gather_ceiling", "gnnpre_plan_destroy", "gnnpre_solve_budget",
+            "gnnpre_plan_status", "gnnpre_inject_alloc_failure", "gnnpre_gather_ceiling", "gnnpre_describe_panels", "gnnpre_plan_destroy", "gnnpre_solve_budget",
             "gnnpre_status_string", "gnnpre_last_cuda_error"]

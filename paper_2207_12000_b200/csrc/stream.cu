@@ -492,6 +492,28 @@ int run_panels(gnnpre_plan* P, const float* X, int64_t ldx, int32_t K, float* co
 
 }  // namespace
 
+}  // namespace gnnpre
+
+// Host only: see include/gnnpre.h.
+extern "C" int gnnpre_describe_panels(int64_t feat_dim, int64_t slab_width, int32_t K, int32_t* jobs_out, int32_t max_jobs,
+                                      int32_t* num_slabs_out, int32_t* num_jobs_out) {
+    if (feat_dim < 32 || feat_dim % 32 != 0 || feat_dim > (1 << 20) || slab_width < 64 || K < 1 || K > GNNPRE_MAX_HOPS ||
+        !num_slabs_out || !num_jobs_out || max_jobs < 0 || (max_jobs > 0 && !jobs_out))
+        return GNNPRE_ERR_INVALID_ARG;
+    const std::vector<gnnpre::Cols> slabs = gnnpre::panel_slabs((int32_t)feat_dim, (int32_t)std::min<int64_t>(slab_width, feat_dim));
+    const std::vector<gnnpre::PanelJob> jobs = gnnpre::panel_jobs(slabs, K);
+    *num_slabs_out = (int32_t)slabs.size();
+    *num_jobs_out = (int32_t)jobs.size();
+    for (size_t i = 0; i < jobs.size() && (int32_t)i < max_jobs; ++i) {
+        const gnnpre::PanelJob& j = jobs[i];
+        const int32_t rec[6] = {j.k, j.lo, j.hi, j.upload, j.drain_lo, j.drain_hi};
+        for (int t = 0; t < 6; ++t) jobs_out[6 * i + t] = rec[t];
+    }
+    return GNNPRE_OK;
+}
+
+namespace gnnpre {
+
 int ensure_streams(gnnpre_plan* P) {
     if (!P->s_h2d) GNNPRE_CUDA(cudaStreamCreateWithFlags(&P->s_h2d, cudaStreamNonBlocking));
     if (!P->s_d2h) GNNPRE_CUDA(cudaStreamCreateWithFlags(&P->s_d2h, cudaStreamNonBlocking));

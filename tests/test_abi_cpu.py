@@ -91,3 +91,42 @@ def test_normalisation_block_count_matches_oracle(binding):
         want = orc.solve_normalisation_blocks(B_A, B_S, B_D, al[0], al[1], al[2], B_GPU, 64)
         got = binding.gnnpre_solve_normalisation_blocks(B_A, B_S, B_D, al[0], al[1], al[2], B_GPU, 64)
         assert got == want, (B_A, B_S, B_D, al, B_GPU)
+
+
+def test_panel_schedule_invariants(binding):
+    """The narrow-first panel schedule of the streamed path, checked as data (no device): the upload slabs tile the
+    columns in order, start 32 wide and never exceed the plan's slab width; walking the jobs in launch order, a hop-1
+    job runs on exactly one upload slab that has been requested, a later hop only reads columns the previous hop has
+    already computed, no job is wider than the slab width (the scratch rows' width), every (hop, column) is computed
+    exactly once and drained exactly once, and nothing is drained before it has been computed."""
+    for F in (128, 160, 256, 512, 1024, 96, 64):
+        for cap in (64, 96, 128, 512):
+            for K in (1, 2, 3, 5):
+                if cap < 64:
+                    continue
+                ns, jobs = binding.gnnpre_describe_panels(F, cap, K)
+                slabs = []
+                for j in jobs:
+                    if j["upload"] >= 0:
+                        assert j["k"] == 1 and j["upload"] == len(slabs)  # uploads are consumed in order
+                        slabs.append((j["lo"], j["hi"]))
+                assert len(slabs) == ns
+                assert slabs[0][0] == 0 and slabs[-1][1] == F
+                assert all(a[1] == b[0] for a, b in zip(slabs, slabs[1:]))
+                assert slabs[0][1] - slabs[0][0] == min(32, F)
+                assert all(0 < hi - lo <= min(cap, F) and lo % 32 == 0 for lo, hi in slabs)
+                computed = np.zeros((K + 1, F), dtype=np.int32)
+                computed[0, :] = 1
+                drained = np.zeros((K + 1, F), dtype=np.int32)
+                for j in jobs:
+                    k, lo, hi = j["k"], j["lo"], j["hi"]
+                    assert 1 <= k <= K and 0 <= lo < hi <= F and hi - lo <= min(cap, F)
+                    assert (computed[k - 1, lo:hi] == 1).all(), (F, cap, K, j)  # its input exists
+                    computed[k, lo:hi] += 1
+                    dl, dh = j["drain_lo"], j["drain_hi"]
+                    if dh > dl:
+                        assert (computed[k, dl:dh] == 1).all(), (F, cap, K, j)  # only finished columns leave
+                        assert dl % 32 == 0  # host pieces start on 128-byte boundaries
+                        drained[k, dl:dh] += 1
+                assert (computed[1:] == 1).all() and (drained[1:] == 1).all(), (F, cap, K)
+    assert binding._lib.gnnpre_describe_panels(100, 64, 2, None, 0, None, None) == -1

@@ -241,3 +241,32 @@ def test_measured_budget_coefficients_agree_with_the_fixed_ones(B):
     assert 1.0 <= r["beta_fixed"] < 3.0, r
     assert r["worst_fit_residual"] < 0.06, r
     assert r["fixed_model_never_below_measured_by_more_than"] < 0.20, r
+
+
+def test_timeline_of_a_streamed_call_is_printed_on_request(B, capfd, monkeypatch):
+    """GNNPRE_LOG=2: the streamed call brackets its copies and compute jobs with timing events and prints the
+    timeline (milliseconds since the call began) to stderr when it ends; results are unchanged."""
+    g = gi.rmat(20000, 160000, 47, directed_candidates=True)
+    F, K = 128, 2
+    X = gi.normal_matrix(g.n, F, 14)
+    plan = B.gnnpre_build_plan(*dev(g), 0, F, operands_mem=B.GNNPRE_MEM_HOST)
+    Xh = X.pin_memory()
+    quiet = [pinned(g.n, F) for _ in range(K)]
+    B.gnnpre_propagate(plan, Xh, K, quiet)
+    capfd.readouterr()
+    monkeypatch.setenv("GNNPRE_LOG", "2")
+    traced = [pinned(g.n, F) for _ in range(K)]
+    B.gnnpre_propagate(plan, Xh, K, traced)
+    err = capfd.readouterr().err
+    lines = [l for l in err.splitlines() if l.startswith("[gnnpre]")]
+    assert sum("h2d X[:, " in l for l in lines) == 3  # the three upload slabs of F = 128
+    assert any("d2h hop 1 cols 0" in l for l in lines) and any("d2h hop 2 cols 64" in l for l in lines)
+    for l in lines:  # "[gnnpre]  <start> ..  <end> ms  <what>": ends do not precede starts
+        t0, t1 = float(l.split()[1]), float(l.split()[3])
+        assert 0.0 <= t0 <= t1
+    for a, b_ in zip(quiet, traced):
+        assert torch.equal(a, b_)
+    monkeypatch.delenv("GNNPRE_LOG")
+    B.gnnpre_propagate(plan, Xh, K, traced)
+    assert "[gnnpre]" not in capfd.readouterr().err
+    plan.close()
