@@ -21,6 +21,9 @@
  *     ordinary process addresses.  The library never takes ownership of a caller's buffer.
  *   - There is no CPU fallback: host-resident operands are streamed through the GPU.
  *   - Only sm_100 devices are accepted (GNNPRE_ERR_UNSUPPORTED_ARCH otherwise).
+ *   - Logging: GNNPRE_LOG=1 in the environment prints one line per gnnpre_propagate call to stderr; GNNPRE_LOG=2
+ *     also prints the timeline of every streamed call (each copy, and the first and last edge block of each
+ *     compute job, in milliseconds since the call began).  Nothing is printed otherwise.
  */
 #ifndef GNNPRE_H
 #define GNNPRE_H

@@ -1,6 +1,7 @@
 // C-ABI glue: argument checks, status text, and the dispatch of gnnpre_propagate.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "gnnpre_internal.cuh"
@@ -91,9 +92,16 @@ extern "C" int gnnpre_propagate(gnnpre_plan_t* P, const float* X, int64_t ldx, i
     GNNPRE_CUDA(cudaGetDevice(&dev));
     if (dev != P->device) return GNNPRE_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (x_mem == GNNPRE_MEM_DEVICE && out_mem == GNNPRE_MEM_DEVICE && P->structure_mem == GNNPRE_MEM_DEVICE)
-        return propagate_resident(P, X, ldx, K, out, ldo, st, stats);
-    return propagate_streamed(P, X, ldx, x_mem, K, out, ldo, out_mem, st, stats);
+    const bool resident = x_mem == GNNPRE_MEM_DEVICE && out_mem == GNNPRE_MEM_DEVICE && P->structure_mem == GNNPRE_MEM_DEVICE;
+    const int rc = resident ? propagate_resident(P, X, ldx, K, out, ldo, st, stats)
+                            : propagate_streamed(P, X, ldx, x_mem, K, out, ldo, out_mem, st, stats);
+    // GNNPRE_LOG >= 1 in the environment: one line per call on stderr (2 adds the timeline of streamed calls)
+    const char* log = std::getenv("GNNPRE_LOG");
+    if (log && std::atoi(log) >= 1)
+        std::fprintf(stderr, "[gnnpre] propagate n=%lld |E|=%lld F=%lld K=%d b=%d c=%d %s -> %s\n", (long long)P->n,
+                     (long long)P->nnz_tilde, (long long)P->feat_dim, K, P->b, P->c,
+                     resident ? "device-resident (enqueued)" : "streamed (complete)", gnnpre_status_string(rc));
+    return rc;
 }
 
 extern "C" int gnnpre_propagate_weighted(gnnpre_plan_t* P, const float* X, int64_t ldx, int32_t K, float* const* out,

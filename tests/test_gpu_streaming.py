@@ -260,8 +260,9 @@ def test_timeline_of_a_streamed_call_is_printed_on_request(B, capfd, monkeypatch
     err = capfd.readouterr().err
     lines = [l for l in err.splitlines() if l.startswith("[gnnpre]")]
     assert sum("h2d X[:, " in l for l in lines) == 3  # the three upload slabs of F = 128
+    assert any("propagate n=20000" in l and "-> ok" in l for l in lines)  # the one-line summary of level 1
     assert any("d2h hop 1 cols 0" in l for l in lines) and any("d2h hop 2 cols 64" in l for l in lines)
-    for l in lines:  # "[gnnpre]  <start> ..  <end> ms  <what>": ends do not precede starts
+    for l in (l for l in lines if " ms  " in l):  # "[gnnpre]  <start> ..  <end> ms  <what>": ends do not precede starts
         t0, t1 = float(l.split()[1]), float(l.split()[3])
         assert 0.0 <= t0 <= t1
     for a, b_ in zip(quiet, traced):
