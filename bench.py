@@ -552,17 +552,28 @@ def c5_streamed_record(B, args):
 
 def configs_object(B, args):
     """Compact records of the other configurations (1, 2, a corner of 3's sweep, and 5 streamed), so that one
-    default run carries a measured line for each of the five."""
+    default run carries a measured line for each of the five.  A record that cannot be taken (say, the host has
+    no room for configuration 5's pinned matrices) reports its error instead of taking the whole run down."""
     import dataclasses
+    import gc
+
+    def attempt(fn, *a, **kw):
+        try:
+            return fn(*a, **kw)
+        except (RuntimeError, MemoryError) as err:  # GnnpreError is a RuntimeError; so are torch's allocation failures
+            gc.collect()
+            torch.cuda.empty_cache()
+            return {"error": f"{type(err).__name__}: {err}"[:300]}
+
     out = {}
-    out["c1"] = compact_resident_record(B, gi.WORKLOADS["c1"], steps=50)
-    out["c2"] = compact_resident_record(B, gi.WORKLOADS["c2"], steps=20)
+    out["c1"] = attempt(compact_resident_record, B, gi.WORKLOADS["c1"], steps=50)
+    out["c2"] = attempt(compact_resident_record, B, gi.WORKLOADS["c2"], steps=20)
     c3 = gi.WORKLOADS["c3"]
     for op, opname in ((gi.OP_GCN, "gcn"), (gi.OP_SAGE, "sage")):
         for F in (16, 128, 512):
-            out[f"c3_{opname}_F{F}"] = compact_resident_record(B, dataclasses.replace(c3, op=op, feat_dim=F), steps=20)
+            out[f"c3_{opname}_F{F}"] = attempt(compact_resident_record, B, dataclasses.replace(c3, op=op, feat_dim=F), steps=20)
     torch.cuda.empty_cache()
-    out["c5"] = c5_streamed_record(B, args)
+    out["c5"] = attempt(c5_streamed_record, B, args)
     return out
 
 
