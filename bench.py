@@ -455,7 +455,7 @@ def time_ceiling(B, plan, X, flush, stream, reps=10):
     return float(np.mean(ms))
 
 
-def compact_resident_record(B, w, steps=20, blocks=None):
+def compact_resident_record(B, w, steps=20, blocks=None, with_cuda_graph=False):
     """One device-resident workload measured like the headline one, reported as a compact record: ms per step
     (all K hops), the segment kernel per hop, and the fetch-only yardstick beside it."""
     g = gi.make_graph(w, device="cuda")
@@ -485,6 +485,15 @@ def compact_resident_record(B, w, steps=20, blocks=None):
            "frac_of_gather_ceiling": ceil_ms / seg_ms_per_hop if seg_ms_per_hop > 0 else None,
            "gather_model_gbs": gather_b / (seg_ms_per_hop * 1e-3) / 1e9,
            "gpu_launches_per_step": t["launches"] / steps}
+    if with_cuda_graph:  # the launch-bound workload also as a replayed CUDA graph of all K hops
+        side = torch.cuda.Stream()
+        side.wait_stream(stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            B.gnnpre_propagate(plan, X, K, outs, stream=side)
+        tg = time_resident(B, plan, X, K, outs, steps, 3, flush, stream, graph=graph)
+        rec["ms_per_step_cuda_graph"] = tg["ms_per_step"]
+        del graph
     plan.close()
     return rec
 
@@ -566,7 +575,7 @@ def configs_object(B, args):
             return {"error": f"{type(err).__name__}: {err}"[:300]}
 
     out = {}
-    out["c1"] = attempt(compact_resident_record, B, gi.WORKLOADS["c1"], steps=50)
+    out["c1"] = attempt(compact_resident_record, B, gi.WORKLOADS["c1"], steps=50, with_cuda_graph=True)
     out["c2"] = attempt(compact_resident_record, B, gi.WORKLOADS["c2"], steps=20)
     c3 = gi.WORKLOADS["c3"]
     for op, opname in ((gi.OP_GCN, "gcn"), (gi.OP_SAGE, "sage")):
