@@ -271,3 +271,31 @@ def test_timeline_of_a_streamed_call_is_printed_on_request(B, capfd, monkeypatch
     B.gnnpre_propagate(plan, Xh, K, traced)
     assert "[gnnpre]" not in capfd.readouterr().err
     plan.close()
+
+
+def test_maximum_hop_count_resident_and_streamed(B):
+    """K = GNNPRE_MAX_HOPS (64) on a small graph under SAGE (a contraction in the max norm, so 64 hops neither grow nor
+    underflow): device-resident, streamed as equal slabs and streamed as panels (65 whole matrices on the device) give
+    the same bits, every hop stays within the tolerance of the un-rounded fp64 chain, and K = 65 is refused."""
+    import oracle as orc
+    from parity_util import TOL, hop_error
+    g = gi.rmat(6000, 60000, 48, directed_candidates=True)
+    F, K = 128, B.GNNPRE_MAX_HOPS
+    X = gi.normal_matrix(g.n, F, 15, device="cuda")
+    plan = B.gnnpre_build_plan(*dev(g), 1, F, force_blocks=2, segment_edges=64)
+    ref, _ = B.gnnpre_propagate(plan, X, K)
+    assert B.gnnpre_plan_status(plan) == 0
+    want = orc.propagate(1, 0.0, g.rowptr.numpy(), g.colidx.numpy(), to_np(X), K)
+    for k in (0, 1, 7, 31, 63):
+        assert hop_error(to_np(ref[k]), want[k]) <= TOL, k
+    with pytest.raises(B.GnnpreError):
+        B.gnnpre_propagate(plan, X, K + 1, [torch.empty_like(X) for _ in range(K + 1)])
+    plan.close()
+    Xh = X.cpu().pin_memory()
+    for kw, schedule in ((dict(force_col_slabs=2), B.GNNPRE_SCHEDULE_SLABS), (dict(), B.GNNPRE_SCHEDULE_PANELS)):
+        hplan = B.gnnpre_build_plan(*dev(g), 1, F, force_blocks=2, segment_edges=64, operands_mem=B.GNNPRE_MEM_HOST, **kw)
+        outs, st = B.gnnpre_propagate(hplan, Xh, K, [pinned(g.n, F) for _ in range(K)], want_stats=True)
+        assert st.schedule == schedule
+        for k in range(K):
+            assert torch.equal(outs[k], ref[k].cpu()), (schedule, k)
+        hplan.close()
