@@ -533,6 +533,7 @@ int propagate_streamed(gnnpre_plan* P, const float* X, int64_t ldx, int32_t x_me
         if (rc == GNNPRE_OK) rc = run_panels(P, X, ldx, K, out, ldo, stream, stats);
         else if (rc == GNNPRE_ERR_OOM_DEVICE) rc = run_slabs(P, X, ldx, x_host, K, out, ldo, out_host, stream, stats);
     } else {
+        for (auto& w : P->whole) w.reset();  // whole matrices kept from an earlier panel call give their room back
         rc = run_slabs(P, X, ldx, x_host, K, out, ldo, out_host, stream, stats);
     }
     if (rc != GNNPRE_OK) {

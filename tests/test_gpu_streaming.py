@@ -299,3 +299,24 @@ def test_maximum_hop_count_resident_and_streamed(B):
         for k in range(K):
             assert torch.equal(outs[k], ref[k].cpu()), (schedule, k)
         hplan.close()
+
+
+def test_schedule_follows_the_hop_count_of_each_call(B):
+    """One plan, three streamed calls: K = 2 fits the budget as whole matrices (panels), K = 6 does not (equal slabs;
+    the whole matrices of the first call are released, so the plan never holds both sets), K = 1 fits again."""
+    g = gi.rmat(20000, 160000, 49, directed_candidates=True)
+    F = 128
+    rp_np, ci_np = g.rowptr.numpy(), g.colidx.numpy()
+    X = gi.normal_matrix(g.n, F, 16)
+    B_X = 4 * g.n * F
+    plan = B.gnnpre_build_plan(*dev(g), 0, F, operands_mem=B.GNNPRE_MEM_HOST)
+    held = plan.info()["device_bytes"]
+    plan.close()
+    plan = B.gnnpre_build_plan(*dev(g), 0, F, operands_mem=B.GNNPRE_MEM_HOST, budget_bytes=held + 5 * B_X)
+    Xh = X.pin_memory()
+    for K, schedule in ((2, B.GNNPRE_SCHEDULE_PANELS), (6, B.GNNPRE_SCHEDULE_SLABS), (1, B.GNNPRE_SCHEDULE_PANELS)):
+        outs, st = B.gnnpre_propagate(plan, Xh, K, [pinned(g.n, F) for _ in range(K)], want_stats=True)
+        assert st.schedule == schedule, K
+        assert plan.info()["device_bytes"] <= held + 5 * B_X
+        check_all_hops(0, 0.0, rp_np, ci_np, X.numpy(), outs)
+    plan.close()
